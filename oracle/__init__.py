@@ -1,0 +1,159 @@
+"""ctypes front end of the CPU oracle (``sirllm_oracle.c``).  TEST INFRASTRUCTURE ONLY.
+
+Nothing on the product path may import this package: it is for the tests, the smoke
+check and the benchmark's CPU-baseline leg.  Arguments are CPU torch tensors (or numpy
+arrays); bf16 / fp16 tensors are passed by their 16-bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sirllm_oracle.c")
+_LIB = os.path.join(_HERE, "libsirllm_oracle.so")
+
+F32, BF16 = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (strict IEEE: no contraction, no fast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math",
+                               "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"])
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+        L.oracle_token_entropy.restype = ctypes.c_double
+        L.oracle_token_entropy.argtypes = [vp, ctypes.c_int, i64, i32, vp]
+        L.oracle_score.restype = ctypes.c_int
+        L.oracle_score.argtypes = [vp, ctypes.c_int, i64, i64, i64, vp, vp]
+        L.oracle_decay.restype = None
+        L.oracle_decay.argtypes = [vp, i64, f32]
+        L.oracle_order_key.restype = ctypes.c_uint32
+        L.oracle_order_key.argtypes = [f32]
+        L.oracle_select.restype = i32
+        L.oracle_select.argtypes = [vp, i32, i32, i32, i32, i32, vp]
+        L.oracle_gather_rows.restype = None
+        L.oracle_gather_rows.argtypes = [vp, vp, i64, vp, i32]
+        L.oracle_step.restype = i32
+        L.oracle_step.argtypes = [vp, i32, vp, vp, vp, i32, f32, i32, i32, i32, i32, i32, vp, vp,
+                                  i64, i64, vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(x):
+    if x is None:
+        return None
+    if isinstance(x, np.ndarray):
+        assert x.flags["C_CONTIGUOUS"]
+        return x.ctypes.data
+    assert x.device.type == "cpu" and x.is_contiguous()
+    return x.data_ptr()
+
+
+def _logits_dtype(logits: torch.Tensor) -> int:
+    if logits.dtype == torch.float32:
+        return F32
+    if logits.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"logits dtype {logits.dtype} not supported")
+
+
+def token_entropy(row: torch.Tensor, token_id: int) -> float:
+    """Token Entropy of one token as a double (before rounding to fp32)."""
+    row = row.contiguous()
+    return lib().oracle_token_entropy(_ptr(row), _logits_dtype(row), row.numel(), int(token_id), None)
+
+
+def score(logits: torch.Tensor, ids: torch.Tensor) -> torch.Tensor:
+    """fp32 scores of the ``T`` rows of ``logits [T, V]`` (last dim contiguous)."""
+    assert logits.dim() == 2 and logits.stride(1) == 1
+    T, V = logits.shape
+    ids = ids.to(torch.int32).contiguous()
+    out = torch.empty(T, dtype=torch.float32)
+    stride = logits.stride(0) if T > 1 else V
+    lib().oracle_score(logits.data_ptr(), _logits_dtype(logits), T, V, stride, _ptr(ids), _ptr(out))
+    return out
+
+
+def decay(E: torch.Tensor, live_len: int, eta: float) -> None:
+    """In place: ``E[:live_len] *= eta`` as single fp32 multiplies."""
+    assert E.dtype == torch.float32
+    lib().oracle_decay(_ptr(E), int(live_len), float(np.float32(eta)))
+
+
+def order_key(x: float) -> int:
+    return lib().oracle_order_key(float(np.float32(x)))
+
+
+def select(E: torch.Tensor, live_len: int, n_sink: int, n_recent: int, budget: int,
+           threshold: int | None = None) -> torch.Tensor:
+    """Kept slots (ascending int32) for scores ``E[:live_len]``."""
+    threshold = budget if threshold is None else threshold
+    assert E.dtype == torch.float32
+    keep = torch.empty(max(int(live_len), budget, 1), dtype=torch.int32)
+    n = lib().oracle_select(_ptr(E), int(live_len), n_sink, n_recent, budget, threshold, _ptr(keep))
+    if n < 0:
+        raise ValueError("inconsistent selection parameters")
+    return keep[:n].clone()
+
+
+def gather_rows(src: torch.Tensor, keep: torch.Tensor) -> torch.Tensor:
+    """``src[keep]`` for a ``[slots, ...]`` tensor, by memcpy of whole rows."""
+    src = src.contiguous()
+    keep = keep.to(torch.int32).contiguous()
+    out = torch.empty((keep.numel(),) + tuple(src.shape[1:]), dtype=src.dtype)
+    row_bytes = src[0].numel() * src.element_size() if src.shape[0] else 0
+    lib().oracle_gather_rows(_ptr(src), _ptr(out), row_bytes, _ptr(keep), keep.numel())
+    return out
+
+
+class Stream:
+    """State of one dialogue stream as the oracle keeps it (Algorithm 1's variables)."""
+
+    def __init__(self, capacity: int, n_sink: int, n_recent: int, budget: int, threshold: int,
+                 eta: float, k: torch.Tensor | None = None, v: torch.Tensor | None = None):
+        self.capacity, self.n_sink, self.n_recent = capacity, n_sink, n_recent
+        self.budget, self.threshold, self.eta = budget, threshold, float(np.float32(eta))
+        self.E = torch.zeros(capacity, dtype=torch.float32)
+        self.serial = torch.full((capacity,), -1, dtype=torch.int64)
+        self.next_serial = ctypes.c_int64(0)
+        self.live_len = 0
+        self.k, self.v = k, v          # [planes, capacity, head_dim] or None
+        self.keep = torch.empty(0, dtype=torch.int32)
+
+    def step(self, new_e: torch.Tensor) -> torch.Tensor:
+        """Append the round's scores (its K/V rows must already sit in the caches), decay,
+        and evict if over the threshold.  Returns the kept-slot list of the round."""
+        new_e = new_e.to(torch.float32).contiguous()
+        T = new_e.numel()
+        keep = torch.empty(max(self.capacity, 1), dtype=torch.int32)
+        n_planes, row_bytes = 0, 0
+        if self.k is not None:
+            assert self.k.is_contiguous() and self.k.shape[1] == self.capacity
+            n_planes = self.k.shape[0]
+            row_bytes = self.k.shape[2] * self.k.element_size()
+        n = lib().oracle_step(_ptr(new_e), T, _ptr(self.E), _ptr(self.serial),
+                              ctypes.addressof(self.next_serial), self.live_len, self.eta,
+                              self.capacity, self.n_sink, self.n_recent, self.budget,
+                              self.threshold, _ptr(self.k), _ptr(self.v), n_planes, row_bytes,
+                              _ptr(keep))
+        if n < 0:
+            raise ValueError("round does not fit the cache or parameters are inconsistent")
+        self.live_len = n
+        self.keep = keep[:n].clone()
+        return self.keep

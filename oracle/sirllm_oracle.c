@@ -1,0 +1,234 @@
+/*
+ * CPU oracle for the SirLLM retention pass.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, single-threaded restatement of what the retention pass computes,
+ * written from the paper (Yao, Li, Zhao: "SirLLM: Streaming Infinite Retentive LLM",
+ * Sections 3.1-3.3 and Algorithm 1).  It exists so that the CUDA library can be
+ * checked against something that is obviously right; it is never part of the
+ * product path, shares no code with it and is only called by the tests, the smoke
+ * check and the benchmark's CPU-baseline leg.
+ *
+ * Arithmetic is double precision wherever arithmetic occurs, except where the
+ * method itself fixes the precision: the entropy cache E is stored as fp32 and the
+ * decay is one fp32 multiply per round (so that repeated decay is reproducible
+ * bit for bit).  Build with -ffp-contract=off and without any fast-math option.
+ *
+ * Every function is pinned by tests/test_oracle_*.py against closed forms, the
+ * paper's printed cache example, brute force on tiny caches, a long-double
+ * recomputation and invariants.  The end-to-end composition (oracle_step) has no
+ * number in the paper to be pinned to beyond those per-part pins: parity unpinned
+ * at the level of whole multi-round streams.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_F32 0
+#define ORACLE_BF16 1
+
+/* ---- reading one logit exactly ------------------------------------------------- */
+
+static double logit_at(const void *row, int dtype, int64_t v)
+{
+    if (dtype == ORACLE_F32)
+        return (double)((const float *)row)[v];
+    /* bfloat16: the upper half of an IEEE binary32 */
+    uint32_t bits = (uint32_t)((const uint16_t *)row)[v] << 16;
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return (double)f;
+}
+
+/*
+ * Token Entropy of one token (Section 3.2, the display equation defining e_i):
+ *     e = -log P(x | context),   P = softmax(z)[x]
+ * with the natural logarithm.  Written as (m - z[x]) + log(sum_v exp(z[v] - m)),
+ * m = max_v z[v]; both addends are >= 0.  A token id of -1 means that no
+ * prediction exists for the position (the first token of a stream) and gives 0.
+ * An id outside [0, V) other than -1 also gives 0 and raises *bad_id.
+ */
+double oracle_token_entropy(const void *row, int dtype, int64_t V, int32_t id, int *bad_id)
+{
+    if (id == -1)
+        return 0.0;
+    if (id < 0 || (int64_t)id >= V) {
+        if (bad_id)
+            *bad_id = 1;
+        return 0.0;
+    }
+    double m = -INFINITY;
+    for (int64_t v = 0; v < V; ++v) {
+        double z = logit_at(row, dtype, v);
+        if (z > m)
+            m = z;
+    }
+    double s = 0.0;
+    for (int64_t v = 0; v < V; ++v)
+        s += exp(logit_at(row, dtype, v) - m);
+    return (m - logit_at(row, dtype, id)) + log(s);
+}
+
+/* Scores of the T tokens of one round (Algorithm 1: E_t = Entropy([I_t, R_t])).
+ * Row t of `logits` (row_stride elements apart) is the distribution token ids[t]
+ * was drawn from.  Returns the number of out-of-range ids. */
+int oracle_score(const void *logits, int dtype, int64_t T, int64_t V, int64_t row_stride,
+                 const int32_t *ids, float *out_e)
+{
+    int n_bad = 0;
+    size_t esz = dtype == ORACLE_F32 ? 4 : 2;
+    for (int64_t t = 0; t < T; ++t) {
+        int bad = 0;
+        const char *row = (const char *)logits + (size_t)t * (size_t)row_stride * esz;
+        out_e[t] = (float)oracle_token_entropy(row, dtype, V, ids[t], &bad);
+        n_bad += bad;
+    }
+    return n_bad;
+}
+
+/* Memory decay (Section 3.3, E = E x eta_decay; Algorithm 1 applies it once per
+ * round, after the round's scores were appended): one fp32 multiply per entry. */
+void oracle_decay(float *E, int64_t l, float eta)
+{
+    for (int64_t i = 0; i < l; ++i) {
+        volatile float p = E[i] * eta; /* volatile: keep the product a rounded fp32 */
+        E[i] = p;
+    }
+}
+
+/* Total order on fp32 bit patterns used to rank scores: larger key = larger score.
+ * Negative values have all bits flipped, non-negative ones the sign bit set. */
+uint32_t oracle_order_key(float x)
+{
+    uint32_t u;
+    memcpy(&u, &x, sizeof u);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+typedef struct {
+    uint32_t key;
+    int32_t slot;
+} ranked_t;
+
+static int by_score_desc_then_slot_asc(const void *pa, const void *pb)
+{
+    const ranked_t *a = pa, *b = pb;
+    if (a->key != b->key)
+        return a->key > b->key ? -1 : 1;
+    return (a->slot > b->slot) - (a->slot < b->slot);
+}
+
+static int by_int_asc(const void *pa, const void *pb)
+{
+    int32_t a = *(const int32_t *)pa, b = *(const int32_t *)pb;
+    return (a > b) - (a < b);
+}
+
+/*
+ * Which slots stay (Sections 3.1 and 3.3; Algorithm 1, the branch taken when the
+ * cache holds more than L tokens).  E[0..l) are the (already decayed) scores.
+ *   l <= threshold : nothing is evicted, keep = 0..l-1.
+ *   otherwise      : keep = sinks [0, n_sink)  U  the k = budget - n_sink - n_recent
+ *                    best-scored slots of the middle [n_sink, l - n_recent)
+ *                    U  recent [l - n_recent, l), listed in ascending slot order.
+ * Ranking in the middle: higher score first, equal scores -> the lower slot first.
+ * Returns the number of kept slots, or -1 on inconsistent parameters.
+ */
+int32_t oracle_select(const float *E, int32_t l, int32_t n_sink, int32_t n_recent, int32_t budget,
+                      int32_t threshold, int32_t *keep)
+{
+    if (l < 0 || n_sink < 0 || n_recent < 0 || budget < n_sink + n_recent || threshold < budget)
+        return -1;
+    if (l <= threshold) {
+        for (int32_t i = 0; i < l; ++i)
+            keep[i] = i;
+        return l;
+    }
+    int32_t lo = n_sink, hi = l - n_recent, k = budget - n_sink - n_recent;
+    int32_t n_mid = hi - lo;
+    ranked_t *mid = malloc(sizeof(ranked_t) * (size_t)(n_mid > 0 ? n_mid : 1));
+    for (int32_t i = lo; i < hi; ++i) {
+        mid[i - lo].key = oracle_order_key(E[i]);
+        mid[i - lo].slot = i;
+    }
+    qsort(mid, (size_t)n_mid, sizeof(ranked_t), by_score_desc_then_slot_asc);
+    int32_t n = 0;
+    for (int32_t i = 0; i < lo; ++i)
+        keep[n++] = i;
+    for (int32_t r = 0; r < k; ++r)
+        keep[n++] = mid[r].slot;
+    for (int32_t i = hi; i < l; ++i)
+        keep[n++] = i;
+    free(mid);
+    qsort(keep, (size_t)n, sizeof(int32_t), by_int_asc);
+    return n;
+}
+
+/* X[Id] of Section 3.1: out[j] = in[keep[j]] for rows of row_bytes bytes, into a
+ * separate output array. */
+void oracle_gather_rows(const void *src, void *dst, int64_t row_bytes, const int32_t *keep,
+                        int32_t n_keep)
+{
+    for (int32_t j = 0; j < n_keep; ++j)
+        memcpy((char *)dst + (size_t)j * (size_t)row_bytes,
+               (const char *)src + (size_t)keep[j] * (size_t)row_bytes, (size_t)row_bytes);
+}
+
+/*
+ * One round of one stream, Algorithm 1 rotated so that the eviction of turn t+1
+ * happens at the end of turn t (the caches the model sees are the same):
+ *   append the round's T scores to E (and serial numbers to `serial`), l += T;
+ *   decay all l scores once; if l > threshold select and compact E, serial and
+ *   every K/V plane; return the new live length.
+ * new_e          [T]  scores of the round's tokens (already computed)
+ * E, serial      [capacity] per-slot score and token serial number, updated in place
+ * k, v           [n_planes, capacity, row_bytes] caches whose slots [l, l+T) already
+ *                hold the round's new rows; compacted in place through a scratch copy
+ * keep           [max(threshold, .)] out: the kept slots (identity when nothing is evicted)
+ * Returns the new live length, or -1 if l + T > capacity (nothing is changed).
+ */
+int32_t oracle_step(const float *new_e, int32_t T, float *E, int64_t *serial, int64_t *next_serial,
+                    int32_t l, float eta, int32_t capacity, int32_t n_sink, int32_t n_recent,
+                    int32_t budget, int32_t threshold, void *k, void *v, int64_t n_planes,
+                    int64_t row_bytes, int32_t *keep)
+{
+    if (l + T > capacity)
+        return -1;
+    for (int32_t t = 0; t < T; ++t) {
+        E[l + t] = new_e[t];
+        if (serial)
+            serial[l + t] = (*next_serial)++;
+    }
+    l += T;
+    oracle_decay(E, l, eta);
+    int32_t n_keep = oracle_select(E, l, n_sink, n_recent, budget, threshold, keep);
+    if (n_keep < 0 || l <= threshold)
+        return n_keep;
+
+    float *E2 = malloc(sizeof(float) * (size_t)n_keep);
+    for (int32_t j = 0; j < n_keep; ++j)
+        E2[j] = E[keep[j]];
+    memcpy(E, E2, sizeof(float) * (size_t)n_keep);
+    free(E2);
+    if (serial) {
+        int64_t *s2 = malloc(sizeof(int64_t) * (size_t)n_keep);
+        for (int32_t j = 0; j < n_keep; ++j)
+            s2[j] = serial[keep[j]];
+        memcpy(serial, s2, sizeof(int64_t) * (size_t)n_keep);
+        free(s2);
+    }
+    size_t kept_bytes = (size_t)n_keep * (size_t)row_bytes;
+    char *tmp = malloc(kept_bytes ? kept_bytes : 1);
+    void *caches[2] = {k, v};
+    for (int c = 0; c < 2; ++c) {
+        if (!caches[c])
+            continue;
+        for (int64_t p = 0; p < n_planes; ++p) {
+            char *plane = (char *)caches[c] + (size_t)p * (size_t)capacity * (size_t)row_bytes;
+            oracle_gather_rows(plane, tmp, row_bytes, keep, n_keep);
+            memcpy(plane, tmp, kept_bytes);
+        }
+    }
+    free(tmp);
+    return n_keep;
+}
