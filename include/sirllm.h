@@ -1,0 +1,179 @@
+/*
+ * sirllm.h - C ABI of the B200 (sm_100a) retention pass of SirLLM
+ * (Yao, Li, Zhao, "SirLLM: Streaming Infinite Retentive LLM").
+ *
+ * One dialogue round of one or more independent streams is
+ *     score  ->  append  ->  decay  ->  select  ->  compact E  ->  compact KV
+ * (Algorithm 1, with the eviction of turn t+1 moved to the end of turn t).  The
+ * calls below expose the three parts and the whole round.
+ *
+ * Conventions shared by every call
+ *   - All data pointers are DEVICE pointers unless an argument is marked (host).
+ *     The library allocates nothing and keeps no device state between calls; the
+ *     caller owns every buffer, including the workspace `ws`
+ *     (sirllm_workspace_bytes() bytes, 256-byte aligned, set up once with
+ *     sirllm_workspace_init()).
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls validate their arguments on the host, enqueue work on that stream and
+ *     return without synchronising (sirllm_status() is the exception).  Two calls
+ *     that use the same workspace must be ordered on the same stream.
+ *   - Return value: SIRLLM_OK or a negative SIRLLM_ERR_* code.  Nothing is
+ *     enqueued when a negative code is returned.  Conditions only the device can
+ *     see are OR-ed into a sticky status word in `ws` (SIRLLM_STATUS_* bits).
+ *   - Layouts.  Logits: row-major rows of `vocab` elements, `logits_row_stride`
+ *     elements apart; stream s owns rows [s*max_new, s*max_new + n_new[s]).
+ *     K and V: each one contiguous array [n_streams][n_layers][n_kv_heads]
+ *     [capacity][head_dim] of 16-bit elements; a "plane" is one [capacity][head_dim]
+ *     slice, a "slot" one row of it.  Scores E: fp32 [n_streams][capacity].
+ *     keep_idx: int32 [n_streams][threshold].  Per-stream scalars: [n_streams].
+ */
+#ifndef SIRLLM_H
+#define SIRLLM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* element types */
+#define SIRLLM_F32 0
+#define SIRLLM_BF16 1
+#define SIRLLM_F16 2
+
+/* return codes */
+#define SIRLLM_OK 0
+#define SIRLLM_ERR_NULL (-1)       /* a required pointer is NULL */
+#define SIRLLM_ERR_BAD_CONFIG (-2) /* inconsistent or unsupported sirllm_config */
+#define SIRLLM_ERR_ALIGN (-3)      /* a pointer or stride breaks the 16-byte alignment rule */
+#define SIRLLM_ERR_CUDA (-4)       /* a CUDA runtime call failed; see sirllm_last_cuda_error() */
+
+/* bits of the device status word */
+#define SIRLLM_STATUS_TOKEN_RANGE 1 /* a token id outside [0, vocab) other than -1; scored 0 */
+#define SIRLLM_STATUS_OVERFLOW 2    /* live_len + n_new > capacity; that stream's round was skipped */
+#define SIRLLM_STATUS_TIMEOUT 4     /* a bounded device-side wait gave up; results are unreliable */
+#define SIRLLM_STATUS_BAD_KEEP 8    /* a caller-supplied keep list is not strictly ascending within
+                                       [0, capacity); that stream was not compacted */
+
+/* Largest `capacity` the selection kernel supports (the scores of one stream are
+ * held in one SM's shared memory). */
+#define SIRLLM_MAX_CAPACITY 49152
+
+typedef struct sirllm_config {
+    int32_t n_streams;   /* independent dialogue streams, >= 1 */
+    int32_t n_layers;    /* K/V planes per stream = n_layers * n_kv_heads (each of K and V) */
+    int32_t n_kv_heads;
+    int32_t head_dim;    /* elements per K/V row; head_dim * 2 bytes must be a multiple of 16 */
+    int32_t capacity;    /* physical slots per plane, <= SIRLLM_MAX_CAPACITY */
+    int32_t budget;      /* retained slots after an eviction = n_sink + n_recent + k  (the
+                            "cache size" of Tables 1-3) */
+    int32_t n_sink;      /* attention-sink slots always kept: the first n_sink (Section 3.1) */
+    int32_t n_recent;    /* most recent slots always kept (Section 3.1; 0 in the SirLLM rows) */
+    int32_t threshold;   /* evict only when live_len > threshold (the L of Algorithm 1);
+                            budget <= threshold <= capacity */
+    int32_t max_new;     /* most tokens one stream appends per round; logits rows per stream */
+    int32_t kv_dtype;    /* SIRLLM_BF16 or SIRLLM_F16 (rows are only copied) */
+    int32_t logits_dtype;/* SIRLLM_F32 or SIRLLM_BF16 */
+    int64_t vocab;       /* V */
+    int64_t logits_row_stride; /* elements between consecutive logits rows, >= vocab */
+} sirllm_config;
+
+/* Bytes of device workspace the calls below need for this configuration (0 if the
+ * configuration is invalid).  Host-only, pure.  No counterpart in the paper. */
+size_t sirllm_workspace_bytes(const sirllm_config *cfg);
+
+/* Zeroes the workspace (status word, scratch).  Call once after allocating it.
+ * No counterpart in the paper. */
+int sirllm_workspace_init(const sirllm_config *cfg, void *ws, void *cuda_stream);
+
+/*
+ * Token Entropy (Section 3.2, the equation defining e_i = -log P(x_i | x_0..x_{i-1}),
+ * natural logarithm): for every stream s and t < n_new[s],
+ *     out_entropy[s*max_new + t] = -log softmax(logits row)[token_ids[s*max_new + t]]
+ * computed as one streaming log-sum-exp over the vocabulary in fp32 (final
+ * combination in fp64).  Row t must be the distribution token t was drawn from; the
+ * library does no shifting.  token id -1 = "no prediction for this position" -> 0.
+ * Any other id outside [0, vocab) -> 0 and SIRLLM_STATUS_TOKEN_RANGE.
+ *   logits      [n_streams*max_new rows] fp32 or bf16, read once, never written
+ *   token_ids   int32 [n_streams*max_new]
+ *   n_new       int32 [n_streams], or NULL meaning max_new for every stream
+ *   out_entropy fp32 [n_streams*max_new]; entries t >= n_new[s] are left untouched
+ * Logits must be finite or -inf, with at least one finite entry per row.
+ */
+int sirllm_score(const sirllm_config *cfg, const void *logits, const int32_t *token_ids,
+                 const int32_t *n_new, float *out_entropy, void *ws, void *cuda_stream);
+
+/*
+ * Memory decay and selection (Section 3.3: E = E x eta_decay, Id_entropy = Top_k(E);
+ * Section 3.1: Id_sink, Id_recent; Algorithm 1's test "KV cache size > L").
+ * For every stream: scores[s][i] <- fp32(scores[s][i] * decay[s]) for i < live_len[s]
+ * (one IEEE multiply, denormals kept); then if live_len[s] <= threshold the keep list
+ * is the identity 0..live_len-1, else it is, in ascending order,
+ *     [0, n_sink)  U  top-k of [n_sink, live_len - n_recent)  U  [live_len - n_recent, live_len)
+ * with k = budget - n_sink - n_recent.  Ranking: higher score first by the total
+ * order on fp32 bit patterns (negatives below positives, -0 < +0); equal scores ->
+ * the lower slot wins.  Exactly one keep list is correct.
+ *   scores   fp32 [n_streams][capacity], updated in place
+ *   serial   int64 [n_streams][capacity] or NULL: an 8-byte tag per slot (e.g. the
+ *            token's text position) that travels with the scores when they are compacted
+ *   live_len int32 [n_streams]; rewritten to n_keep only if compact_scores != 0
+ *   decay    fp32 [n_streams]
+ *   keep_idx int32 [n_streams][threshold] out;  n_keep int32 [n_streams] out
+ *   compact_scores != 0: also scores[s][j] <- scores[s][keep[j]] (and serial), j < n_keep
+ */
+int sirllm_decay_select(const sirllm_config *cfg, float *scores, int64_t *serial, int32_t *live_len,
+                        const float *decay, int32_t *keep_idx, int32_t *n_keep,
+                        int32_t compact_scores, void *ws, void *cuda_stream);
+
+/*
+ * KV gather (Section 3.1, X[Id]; Section 3.3, KV_cache = KV_cache[Id_sink, Id_entropy]):
+ * for every plane p of stream s and j < n_keep[s]:  dst[p][j][:] <- src[p][keep_idx[s][j]][:].
+ * Rows keep their relative order, so slot order = order in the text (the positions
+ * example of Section 3.3).  k_dst == k_src (and v_dst == v_src) compacts in place;
+ * otherwise source and destination must not overlap.  Either of K or V may be NULL
+ * (both src and dst) to skip it.  Every keep list must be strictly ascending within
+ * [0, capacity) (else SIRLLM_STATUS_BAD_KEEP and the stream is left alone).
+ */
+int sirllm_compact_kv(const sirllm_config *cfg, const void *k_src, const void *v_src, void *k_dst,
+                      void *v_dst, const int32_t *keep_idx, const int32_t *n_keep, void *ws,
+                      void *cuda_stream);
+
+/*
+ * One whole round (Algorithm 1's loop body): score the n_new[s] new tokens, append
+ * their scores at scores[s][live_len[s] ...] (their K/V rows and serial tags must
+ * already sit in slots [live_len[s], live_len[s] + n_new[s]) of every plane), decay
+ * all scores once, and if the new length exceeds `threshold` select, compact the
+ * scores (and tags) and compact K and V in place.  live_len[s] becomes the new
+ * length.  If live_len[s] + n_new[s] > capacity the stream is skipped untouched and
+ * SIRLLM_STATUS_OVERFLOW is raised.
+ *   keep_idx, n_keep  out as in sirllm_decay_select
+ *   new_entropy       fp32 [n_streams*max_new] out or NULL: the raw (undecayed) scores
+ */
+int sirllm_step(const sirllm_config *cfg, const void *logits, const int32_t *token_ids,
+                const int32_t *n_new, float *scores, int64_t *serial, int32_t *live_len,
+                const float *decay, void *k, void *v, int32_t *keep_idx, int32_t *n_keep,
+                float *new_entropy, void *ws, void *cuda_stream);
+
+/* sirllm_step with four caller-created cudaEvent_t handles (host array phase_events[4])
+ * recorded on the stream before scoring, before selection, before KV compaction and
+ * after it, so that a profiler-free caller can time the three phases.  The work done is
+ * identical to sirllm_step.  No counterpart in the paper. */
+int sirllm_step_phases(const sirllm_config *cfg, const void *logits, const int32_t *token_ids,
+                       const int32_t *n_new, float *scores, int64_t *serial, int32_t *live_len,
+                       const float *decay, void *k, void *v, int32_t *keep_idx, int32_t *n_keep,
+                       float *new_entropy, void *ws, void *cuda_stream, void **phase_events);
+
+/* Waits for the stream, copies the status word to *status_out (host) and, if
+ * `clear` != 0, resets it.  No counterpart in the paper. */
+int sirllm_status(void *ws, void *cuda_stream, int32_t *status_out, int32_t clear);
+
+/* Text for a return code; the message of the last failed CUDA call of this thread.
+ * No counterpart in the paper. */
+const char *sirllm_strerror(int code);
+const char *sirllm_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SIRLLM_H */

@@ -1,0 +1,240 @@
+"""ctypes binding of ``libsirllm.so``: same names as the C ABI, argument marshalling only.
+
+Every function takes CUDA torch tensors (device memory owned by the caller), checks
+dtypes and contiguity, passes raw pointers and the current CUDA stream to the library
+and raises :class:`SirllmError` on a negative return code.  There is no CPU fallback:
+if the library is missing or a tensor is not on a CUDA device the call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libsirllm.so")
+
+F32, BF16, F16 = 0, 1, 2
+OK, ERR_NULL, ERR_BAD_CONFIG, ERR_ALIGN, ERR_CUDA = 0, -1, -2, -3, -4
+STATUS_TOKEN_RANGE, STATUS_OVERFLOW, STATUS_TIMEOUT, STATUS_BAD_KEEP = 1, 2, 4, 8
+MAX_CAPACITY = 49152
+
+EXPORTS = ["sirllm_workspace_bytes", "sirllm_workspace_init", "sirllm_score", "sirllm_decay_select",
+           "sirllm_compact_kv", "sirllm_step", "sirllm_step_phases", "sirllm_status", "sirllm_strerror",
+           "sirllm_last_cuda_error"]
+
+_DTYPE_CODE = {torch.float32: F32, torch.bfloat16: BF16, torch.float16: F16}
+
+
+class SirllmError(RuntimeError):
+    def __init__(self, code: int, detail: str = ""):
+        self.code = code
+        super().__init__(f"sirllm error {code}: {detail}")
+
+
+class Config(ctypes.Structure):
+    """Mirror of ``sirllm_config``."""
+    _fields_ = [("n_streams", ctypes.c_int32), ("n_layers", ctypes.c_int32),
+                ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("capacity", ctypes.c_int32), ("budget", ctypes.c_int32),
+                ("n_sink", ctypes.c_int32), ("n_recent", ctypes.c_int32),
+                ("threshold", ctypes.c_int32), ("max_new", ctypes.c_int32),
+                ("kv_dtype", ctypes.c_int32), ("logits_dtype", ctypes.c_int32),
+                ("vocab", ctypes.c_int64), ("logits_row_stride", ctypes.c_int64)]
+
+    @property
+    def planes_per_stream(self) -> int:
+        return self.n_layers * self.n_kv_heads
+
+
+def make_config(n_streams, n_layers, n_kv_heads, head_dim, capacity, budget, n_sink, n_recent,
+                max_new, vocab, logits_dtype, kv_dtype, threshold=None, logits_row_stride=None) -> Config:
+    code = lambda d: _DTYPE_CODE[d] if isinstance(d, torch.dtype) else {"f32": F32, "bf16": BF16, "f16": F16}[d]
+    return Config(n_streams, n_layers, n_kv_heads, head_dim, capacity, budget, n_sink, n_recent,
+                  budget if threshold is None else threshold, max_new, code(kv_dtype),
+                  code(logits_dtype), vocab, vocab if logits_row_stride is None else logits_row_stride)
+
+
+def config_from_workload(w, **overrides) -> Config:
+    """Config for a :class:`workloads.Workload`."""
+    kw = dict(n_streams=w.n_streams, n_layers=w.n_layers, n_kv_heads=w.n_kv_heads,
+              head_dim=w.head_dim, capacity=w.capacity, budget=w.budget, n_sink=w.n_sink,
+              n_recent=w.n_recent, max_new=w.new_tokens, vocab=w.vocab,
+              logits_dtype=w.logits_dtype, kv_dtype=w.kv_dtype, threshold=w.threshold)
+    kw.update(overrides)
+    return make_config(**kw)
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library; raises if it was not built (``python -m paper_2405_12528_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise SirllmError(ERR_CUDA, f"{_LIB_PATH} not built; run paper_2405_12528_b200/build.py")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i32, cfgp = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(Config)
+        L.sirllm_workspace_bytes.restype = ctypes.c_size_t
+        L.sirllm_workspace_bytes.argtypes = [cfgp]
+        L.sirllm_workspace_init.restype = ctypes.c_int
+        L.sirllm_workspace_init.argtypes = [cfgp, vp, vp]
+        L.sirllm_score.restype = ctypes.c_int
+        L.sirllm_score.argtypes = [cfgp, vp, vp, vp, vp, vp, vp]
+        L.sirllm_decay_select.restype = ctypes.c_int
+        L.sirllm_decay_select.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, i32, vp, vp]
+        L.sirllm_compact_kv.restype = ctypes.c_int
+        L.sirllm_compact_kv.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.sirllm_step.restype = ctypes.c_int
+        L.sirllm_step.argtypes = [cfgp] + [vp] * 14
+        L.sirllm_step_phases.restype = ctypes.c_int
+        L.sirllm_step_phases.argtypes = [cfgp] + [vp] * 14 + [ctypes.POINTER(vp)]
+        L.sirllm_status.restype = ctypes.c_int
+        L.sirllm_status.argtypes = [vp, vp, ctypes.POINTER(i32), i32]
+        L.sirllm_strerror.restype = ctypes.c_char_p
+        L.sirllm_strerror.argtypes = [ctypes.c_int]
+        L.sirllm_last_cuda_error.restype = ctypes.c_char_p
+        L.sirllm_last_cuda_error.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _check(rc: int) -> None:
+    if rc != OK:
+        L = lib()
+        detail = L.sirllm_strerror(rc).decode()
+        if rc == ERR_CUDA:
+            detail += ": " + L.sirllm_last_cuda_error().decode()
+        raise SirllmError(rc, detail)
+
+
+def _dev(t: Optional[torch.Tensor], dtype=None, name="tensor") -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise SirllmError(ERR_NULL, f"{name} must be a CUDA tensor (there is no CPU path)")
+    if not t.is_contiguous():
+        raise SirllmError(ERR_ALIGN, f"{name} must be contiguous")
+    if dtype is not None and t.dtype not in (dtype if isinstance(dtype, tuple) else (dtype,)):
+        raise SirllmError(ERR_BAD_CONFIG, f"{name} has dtype {t.dtype}")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _logits_ptr(cfg: Config, logits: torch.Tensor) -> int:
+    if not logits.is_cuda:
+        raise SirllmError(ERR_NULL, "logits must be a CUDA tensor (there is no CPU path)")
+    if _DTYPE_CODE.get(logits.dtype) != cfg.logits_dtype:
+        raise SirllmError(ERR_BAD_CONFIG, f"logits dtype {logits.dtype} does not match the config")
+    if logits.stride(-1) != 1 or (logits.dim() >= 2 and logits.shape[-2] > 1
+                                  and logits.stride(-2) != cfg.logits_row_stride):
+        raise SirllmError(ERR_ALIGN, "logits rows must be logits_row_stride elements apart")
+    return logits.data_ptr()
+
+
+def sirllm_workspace_bytes(cfg: Config) -> int:
+    return lib().sirllm_workspace_bytes(ctypes.byref(cfg))
+
+
+def new_workspace(cfg: Config, device="cuda") -> torch.Tensor:
+    """Allocates (with torch) and initialises a workspace for ``cfg``."""
+    n = sirllm_workspace_bytes(cfg)
+    if n == 0:
+        raise SirllmError(ERR_BAD_CONFIG, "invalid configuration")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    sirllm_workspace_init(cfg, ws)
+    return ws
+
+
+def sirllm_workspace_init(cfg: Config, ws: torch.Tensor) -> None:
+    _check(lib().sirllm_workspace_init(ctypes.byref(cfg), _dev(ws, torch.uint8, "ws"), _stream()))
+
+
+def sirllm_score(cfg: Config, logits, token_ids, n_new, out_entropy, ws) -> None:
+    _check(lib().sirllm_score(ctypes.byref(cfg), _logits_ptr(cfg, logits),
+                              _dev(token_ids, torch.int32, "token_ids"),
+                              _dev(n_new, torch.int32, "n_new"),
+                              _dev(out_entropy, torch.float32, "out_entropy"),
+                              _dev(ws, torch.uint8, "ws"), _stream()))
+
+
+def sirllm_decay_select(cfg: Config, scores, serial, live_len, decay, keep_idx, n_keep,
+                        compact_scores, ws) -> None:
+    _check(lib().sirllm_decay_select(ctypes.byref(cfg), _dev(scores, torch.float32, "scores"),
+                                     _dev(serial, torch.int64, "serial"),
+                                     _dev(live_len, torch.int32, "live_len"),
+                                     _dev(decay, torch.float32, "decay"),
+                                     _dev(keep_idx, torch.int32, "keep_idx"),
+                                     _dev(n_keep, torch.int32, "n_keep"),
+                                     int(bool(compact_scores)), _dev(ws, torch.uint8, "ws"), _stream()))
+
+
+_KV = (torch.bfloat16, torch.float16)
+
+
+def sirllm_compact_kv(cfg: Config, k_src, v_src, k_dst, v_dst, keep_idx, n_keep, ws) -> None:
+    _check(lib().sirllm_compact_kv(ctypes.byref(cfg), _dev(k_src, _KV, "k_src"), _dev(v_src, _KV, "v_src"),
+                                   _dev(k_dst, _KV, "k_dst"), _dev(v_dst, _KV, "v_dst"),
+                                   _dev(keep_idx, torch.int32, "keep_idx"),
+                                   _dev(n_keep, torch.int32, "n_keep"),
+                                   _dev(ws, torch.uint8, "ws"), _stream()))
+
+
+def sirllm_step(cfg: Config, logits, token_ids, n_new, scores, serial, live_len, decay, k, v,
+                keep_idx, n_keep, new_entropy, ws) -> None:
+    _check(lib().sirllm_step(ctypes.byref(cfg), _logits_ptr(cfg, logits),
+                             _dev(token_ids, torch.int32, "token_ids"),
+                             _dev(n_new, torch.int32, "n_new"),
+                             _dev(scores, torch.float32, "scores"),
+                             _dev(serial, torch.int64, "serial"),
+                             _dev(live_len, torch.int32, "live_len"),
+                             _dev(decay, torch.float32, "decay"),
+                             _dev(k, _KV, "k"), _dev(v, _KV, "v"),
+                             _dev(keep_idx, torch.int32, "keep_idx"),
+                             _dev(n_keep, torch.int32, "n_keep"),
+                             _dev(new_entropy, torch.float32, "new_entropy"),
+                             _dev(ws, torch.uint8, "ws"), _stream()))
+
+
+def sirllm_step_phases(cfg: Config, logits, token_ids, n_new, scores, serial, live_len, decay, k, v,
+                       keep_idx, n_keep, new_entropy, ws, events) -> None:
+    """``sirllm_step`` that records the four ``torch.cuda.Event`` objects in ``events``
+    (created with ``enable_timing=True``) around its three phases."""
+    handles = (ctypes.c_void_p * 4)()
+    for i, ev in enumerate(events):
+        if not ev.cuda_event:          # torch creates the handle lazily, on first record
+            ev.record()
+        handles[i] = ev.cuda_event
+    _check(lib().sirllm_step_phases(ctypes.byref(cfg), _logits_ptr(cfg, logits),
+                                    _dev(token_ids, torch.int32, "token_ids"),
+                                    _dev(n_new, torch.int32, "n_new"),
+                                    _dev(scores, torch.float32, "scores"),
+                                    _dev(serial, torch.int64, "serial"),
+                                    _dev(live_len, torch.int32, "live_len"),
+                                    _dev(decay, torch.float32, "decay"),
+                                    _dev(k, _KV, "k"), _dev(v, _KV, "v"),
+                                    _dev(keep_idx, torch.int32, "keep_idx"),
+                                    _dev(n_keep, torch.int32, "n_keep"),
+                                    _dev(new_entropy, torch.float32, "new_entropy"),
+                                    _dev(ws, torch.uint8, "ws"), _stream(), handles))
+
+
+def sirllm_status(ws: torch.Tensor, clear: bool = False) -> int:
+    """Synchronises the current stream and returns the device status word."""
+    out = ctypes.c_int32(0)
+    _check(lib().sirllm_status(_dev(ws, torch.uint8, "ws"), _stream(), ctypes.byref(out), int(clear)))
+    return out.value
+
+
+def sirllm_strerror(code: int) -> str:
+    return lib().sirllm_strerror(code).decode()
+
+
+def sirllm_last_cuda_error() -> str:
+    return lib().sirllm_last_cuda_error().decode()

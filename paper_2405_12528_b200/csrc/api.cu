@@ -1,0 +1,285 @@
+// Host side of the C ABI declared in sirllm.h: argument checks, workspace layout and
+// the launch sequences.  No device memory is allocated here.
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace sirllm {
+
+static thread_local char g_cuda_msg[256] = "";
+
+static int cuda_fail(cudaError_t e, const char* where) {
+    snprintf(g_cuda_msg, sizeof g_cuda_msg, "%s: %s", where, cudaGetErrorString(e));
+    return SIRLLM_ERR_CUDA;
+}
+
+int validate_config(const sirllm_config* c) {
+    if (c == nullptr) return SIRLLM_ERR_NULL;
+    if (c->n_streams < 1 || c->n_layers < 1 || c->n_kv_heads < 1 || c->head_dim < 1)
+        return SIRLLM_ERR_BAD_CONFIG;
+    if (c->capacity < 1 || c->capacity > SIRLLM_MAX_CAPACITY) return SIRLLM_ERR_BAD_CONFIG;
+    if (c->n_sink < 0 || c->n_recent < 0 || c->budget < c->n_sink + c->n_recent)
+        return SIRLLM_ERR_BAD_CONFIG;
+    if (c->budget < 1 || c->threshold < c->budget || c->capacity < c->threshold)
+        return SIRLLM_ERR_BAD_CONFIG;
+    if (c->max_new < 0 || c->max_new > c->capacity) return SIRLLM_ERR_BAD_CONFIG;
+    if (c->kv_dtype != SIRLLM_BF16 && c->kv_dtype != SIRLLM_F16) return SIRLLM_ERR_BAD_CONFIG;
+    if (c->logits_dtype != SIRLLM_F32 && c->logits_dtype != SIRLLM_BF16)
+        return SIRLLM_ERR_BAD_CONFIG;
+    if (c->vocab < 1 || c->vocab > 0x7FFFFFFF || c->logits_row_stride < c->vocab)
+        return SIRLLM_ERR_BAD_CONFIG;
+    if ((int64_t)c->head_dim * 2 % 16 != 0 || (int64_t)c->head_dim * 2 > 4096)
+        return SIRLLM_ERR_BAD_CONFIG;
+    if ((int64_t)c->n_streams * c->n_layers * c->n_kv_heads > 0x3FFFFFFF)
+        return SIRLLM_ERR_BAD_CONFIG;
+    return SIRLLM_OK;
+}
+
+WorkspaceLayout workspace_layout(const sirllm_config& c) {
+    WorkspaceLayout L;
+    const int64_t epv = 16 / logits_elem_bytes(c.logits_dtype);
+    const int64_t nvec = c.vocab / epv;
+    L.n_seg = (int32_t)((nvec + kVecPerSeg - 1) / kVecPerSeg);
+    if (L.n_seg < 1) L.n_seg = 1;
+    size_t off = 256;
+    L.first_moved_off = off;
+    off = align_up(off + (size_t)c.n_streams * 4, 256);
+    L.n_keep_off = off;
+    off = align_up(off + (size_t)c.n_streams * 4, 256);
+    L.keep_off = off;
+    off = align_up(off + (size_t)c.n_streams * c.threshold * 4, 256);
+    L.partials_off = off;
+    off = align_up(off + (size_t)c.n_streams * c.max_new * L.n_seg * sizeof(float2), 256);
+    L.total = off;
+    return L;
+}
+
+static bool misaligned(const void* p, size_t a) { return ((uintptr_t)p % a) != 0; }
+
+static ScoreParams score_params(const sirllm_config& c, const WorkspaceLayout& L, const void* logits,
+                                const int32_t* ids, const int32_t* n_new, void* ws) {
+    ScoreParams sp;
+    sp.logits = logits;
+    sp.token_ids = ids;
+    sp.n_new = n_new;
+    sp.partials = (float2*)((char*)ws + L.partials_off);
+    sp.vocab = c.vocab;
+    sp.row_stride = c.logits_row_stride;
+    sp.n_streams = c.n_streams;
+    sp.max_new = c.max_new;
+    sp.n_seg = L.n_seg;
+    sp.logits_dtype = c.logits_dtype;
+    return sp;
+}
+
+static int check_logits(const sirllm_config& c, const void* logits) {
+    if (misaligned(logits, logits_elem_bytes(c.logits_dtype))) return SIRLLM_ERR_ALIGN;
+    return SIRLLM_OK;
+}
+
+}  // namespace sirllm
+
+using namespace sirllm;
+
+extern "C" {
+
+size_t sirllm_workspace_bytes(const sirllm_config* cfg) {
+    if (validate_config(cfg) != SIRLLM_OK) return 0;
+    return workspace_layout(*cfg).total;
+}
+
+int sirllm_workspace_init(const sirllm_config* cfg, void* ws, void* cuda_stream) {
+    int rc = validate_config(cfg);
+    if (rc != SIRLLM_OK) return rc;
+    if (ws == nullptr) return SIRLLM_ERR_NULL;
+    if (misaligned(ws, 256)) return SIRLLM_ERR_ALIGN;
+    cudaError_t e = cudaMemsetAsync(ws, 0, workspace_layout(*cfg).total, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "cudaMemsetAsync");
+}
+
+int sirllm_score(const sirllm_config* cfg, const void* logits, const int32_t* token_ids,
+                 const int32_t* n_new, float* out_entropy, void* ws, void* cuda_stream) {
+    int rc = validate_config(cfg);
+    if (rc != SIRLLM_OK) return rc;
+    if (!logits || !token_ids || !out_entropy || !ws) return SIRLLM_ERR_NULL;
+    if (misaligned(ws, 256)) return SIRLLM_ERR_ALIGN;
+    if ((rc = check_logits(*cfg, logits)) != SIRLLM_OK) return rc;
+    const WorkspaceLayout L = workspace_layout(*cfg);
+    const ScoreParams sp = score_params(*cfg, L, logits, token_ids, n_new, ws);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = launch_score_partials(sp, st);
+    if (e != cudaSuccess) return cuda_fail(e, "score_partials");
+    e = launch_score_finalize(sp, out_entropy, (int32_t*)ws, st);
+    if (e != cudaSuccess) return cuda_fail(e, "score_finalize");
+    return SIRLLM_OK;
+}
+
+static SelectParams select_params(const sirllm_config& c, const WorkspaceLayout& L, float* scores,
+                                  int64_t* serial, int32_t* live_len, const float* decay,
+                                  int32_t* keep_idx, int32_t* n_keep, void* ws) {
+    SelectParams p;
+    memset(&p, 0, sizeof p);
+    p.scores = scores;
+    p.serial = serial;
+    p.live_len = live_len;
+    p.decay = decay;
+    p.keep_idx = keep_idx ? keep_idx : (int32_t*)((char*)ws + L.keep_off);
+    p.n_keep = n_keep ? n_keep : (int32_t*)((char*)ws + L.n_keep_off);
+    p.first_moved = (int32_t*)((char*)ws + L.first_moved_off);
+    p.status = (int32_t*)ws;
+    p.capacity = c.capacity;
+    p.budget = c.budget;
+    p.n_sink = c.n_sink;
+    p.n_recent = c.n_recent;
+    p.threshold = c.threshold;
+    return p;
+}
+
+int sirllm_decay_select(const sirllm_config* cfg, float* scores, int64_t* serial, int32_t* live_len,
+                        const float* decay, int32_t* keep_idx, int32_t* n_keep,
+                        int32_t compact_scores, void* ws, void* cuda_stream) {
+    int rc = validate_config(cfg);
+    if (rc != SIRLLM_OK) return rc;
+    if (!scores || !live_len || !decay || !keep_idx || !n_keep || !ws) return SIRLLM_ERR_NULL;
+    if (misaligned(ws, 256)) return SIRLLM_ERR_ALIGN;
+    const WorkspaceLayout L = workspace_layout(*cfg);
+    SelectParams p = select_params(*cfg, L, scores, serial, live_len, decay, keep_idx, n_keep, ws);
+    p.compact_scores = compact_scores != 0;
+    p.score_new = 0;
+    cudaError_t e = launch_select(p, cfg->n_streams, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "select");
+}
+
+static int compact_params(const sirllm_config& c, const WorkspaceLayout& L, const void* k_src,
+                          const void* v_src, void* k_dst, void* v_dst, const int32_t* keep_idx,
+                          const int32_t* n_keep, void* ws, CompactParams* out) {
+    if ((k_src == nullptr) != (k_dst == nullptr) || (v_src == nullptr) != (v_dst == nullptr))
+        return SIRLLM_ERR_NULL;
+    const void* ptrs[4] = {k_src, v_src, k_dst, v_dst};
+    for (const void* q : ptrs)
+        if (q && misaligned(q, 16)) return SIRLLM_ERR_ALIGN;
+    CompactParams p;
+    memset(&p, 0, sizeof p);
+    p.src[0] = (const char*)k_src;
+    p.src[1] = (const char*)v_src;
+    p.dst[0] = (char*)k_dst;
+    p.dst[1] = (char*)v_dst;
+    p.keep_idx = keep_idx;
+    p.n_keep = n_keep;
+    p.first_moved = (int32_t*)((char*)ws + L.first_moved_off);
+    p.status = (int32_t*)ws;
+    p.planes_per_stream = c.n_layers * c.n_kv_heads;
+    p.planes_per_tensor = (int64_t)c.n_streams * p.planes_per_stream;
+    p.capacity = c.capacity;
+    p.keep_stride = c.threshold;
+    p.row_bytes = c.head_dim * 2;
+    const bool k_in = k_src && k_src == k_dst, v_in = v_src && v_src == v_dst;
+    const bool k_out = k_src && k_src != k_dst, v_out = v_src && v_src != v_dst;
+    if ((k_in || v_in) && (k_out || v_out)) return SIRLLM_ERR_BAD_CONFIG;  // do not mix modes
+    p.in_place = (k_in || v_in) ? 1 : 0;
+    *out = p;
+    return SIRLLM_OK;
+}
+
+int sirllm_compact_kv(const sirllm_config* cfg, const void* k_src, const void* v_src, void* k_dst,
+                      void* v_dst, const int32_t* keep_idx, const int32_t* n_keep, void* ws,
+                      void* cuda_stream) {
+    int rc = validate_config(cfg);
+    if (rc != SIRLLM_OK) return rc;
+    if (!keep_idx || !n_keep || !ws) return SIRLLM_ERR_NULL;
+    if (misaligned(ws, 256)) return SIRLLM_ERR_ALIGN;
+    const WorkspaceLayout L = workspace_layout(*cfg);
+    CompactParams p;
+    if ((rc = compact_params(*cfg, L, k_src, v_src, k_dst, v_dst, keep_idx, n_keep, ws, &p)) != SIRLLM_OK)
+        return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = launch_compact_plan(p, cfg->n_streams, (int32_t*)((char*)ws + L.first_moved_off), st);
+    if (e != cudaSuccess) return cuda_fail(e, "compact_plan");
+    e = launch_compact(p, st);
+    return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "compact");
+}
+
+static int step_impl(const sirllm_config* cfg, const void* logits, const int32_t* token_ids,
+                     const int32_t* n_new, float* scores, int64_t* serial, int32_t* live_len,
+                     const float* decay, void* k, void* v, int32_t* keep_idx, int32_t* n_keep,
+                     float* new_entropy, void* ws, void* cuda_stream, void** ev) {
+    int rc = validate_config(cfg);
+    if (rc != SIRLLM_OK) return rc;
+    if (!logits || !token_ids || !scores || !live_len || !decay || !ws) return SIRLLM_ERR_NULL;
+    if (misaligned(ws, 256)) return SIRLLM_ERR_ALIGN;
+    if ((rc = check_logits(*cfg, logits)) != SIRLLM_OK) return rc;
+    const WorkspaceLayout L = workspace_layout(*cfg);
+    SelectParams sp = select_params(*cfg, L, scores, serial, live_len, decay, keep_idx, n_keep, ws);
+    sp.sc = score_params(*cfg, L, logits, token_ids, n_new, ws);
+    sp.new_entropy = new_entropy;
+    sp.compact_scores = 1;
+    sp.score_new = 1;
+    CompactParams cp;
+    if ((rc = compact_params(*cfg, L, k, v, k, v, sp.keep_idx, sp.n_keep, ws, &cp)) != SIRLLM_OK)
+        return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e;
+#define SIRLLM_MARK(i)                                                        \
+    if (ev && (e = cudaEventRecord((cudaEvent_t)ev[i], st)) != cudaSuccess) \
+        return cuda_fail(e, "cudaEventRecord");
+    SIRLLM_MARK(0)
+    e = launch_score_partials(sp.sc, st);
+    if (e != cudaSuccess) return cuda_fail(e, "score_partials");
+    SIRLLM_MARK(1)
+    e = launch_select(sp, cfg->n_streams, st);
+    if (e != cudaSuccess) return cuda_fail(e, "select");
+    SIRLLM_MARK(2)
+    e = launch_compact(cp, st);
+    if (e != cudaSuccess) return cuda_fail(e, "compact");
+    SIRLLM_MARK(3)
+#undef SIRLLM_MARK
+    return SIRLLM_OK;
+}
+
+int sirllm_step(const sirllm_config* cfg, const void* logits, const int32_t* token_ids,
+                const int32_t* n_new, float* scores, int64_t* serial, int32_t* live_len,
+                const float* decay, void* k, void* v, int32_t* keep_idx, int32_t* n_keep,
+                float* new_entropy, void* ws, void* cuda_stream) {
+    return step_impl(cfg, logits, token_ids, n_new, scores, serial, live_len, decay, k, v, keep_idx,
+                     n_keep, new_entropy, ws, cuda_stream, nullptr);
+}
+
+int sirllm_step_phases(const sirllm_config* cfg, const void* logits, const int32_t* token_ids,
+                       const int32_t* n_new, float* scores, int64_t* serial, int32_t* live_len,
+                       const float* decay, void* k, void* v, int32_t* keep_idx, int32_t* n_keep,
+                       float* new_entropy, void* ws, void* cuda_stream, void** phase_events) {
+    if (!phase_events) return SIRLLM_ERR_NULL;
+    for (int i = 0; i < 4; ++i)
+        if (!phase_events[i]) return SIRLLM_ERR_NULL;
+    return step_impl(cfg, logits, token_ids, n_new, scores, serial, live_len, decay, k, v, keep_idx,
+                     n_keep, new_entropy, ws, cuda_stream, phase_events);
+}
+
+int sirllm_status(void* ws, void* cuda_stream, int32_t* status_out, int32_t clear) {
+    if (!ws || !status_out) return SIRLLM_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMemcpyAsync(status_out, ws, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync");
+    if (clear) {
+        e = cudaMemsetAsync(ws, 0, sizeof(int32_t), st);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+    }
+    e = cudaStreamSynchronize(st);
+    return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "cudaStreamSynchronize");
+}
+
+const char* sirllm_strerror(int code) {
+    switch (code) {
+        case SIRLLM_OK: return "ok";
+        case SIRLLM_ERR_NULL: return "a required pointer is NULL";
+        case SIRLLM_ERR_BAD_CONFIG: return "inconsistent or unsupported configuration";
+        case SIRLLM_ERR_ALIGN: return "pointer or stride not aligned as required";
+        case SIRLLM_ERR_CUDA: return "CUDA runtime error (see sirllm_last_cuda_error)";
+        default: return "unknown error code";
+    }
+}
+
+const char* sirllm_last_cuda_error(void) { return g_cuda_msg; }
+
+}  // extern "C"

@@ -1,0 +1,121 @@
+// Internal declarations shared by the kernels of the retention pass (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sirllm.h"
+
+namespace sirllm {
+
+// ---- workspace layout (device memory owned by the caller) -------------------------------
+//   [0, 256)                              header: int32 status word
+//   first_moved[n_streams]                first slot whose row changes place when compacting
+//   n_keep_fallback[n_streams]            used when the caller passes no n_keep
+//   keep_fallback[n_streams][threshold]   used when the caller passes no keep_idx
+//   partials[n_streams*max_new][n_seg]    (scaled max, sum) pairs of the split log-sum-exp
+struct WorkspaceLayout {
+    size_t first_moved_off;
+    size_t n_keep_off;
+    size_t keep_off;
+    size_t partials_off;
+    size_t total;
+    int32_t n_seg;  // vocabulary segments per logits row
+};
+
+constexpr int kVecPerSeg = 512;  // 16-byte vectors per segment: 8 KB of logits per warp
+constexpr int kScoreWarpsPerCta = 8;
+constexpr int kSelectThreads = 1024;
+constexpr int kRadixBits = 11;
+constexpr int kRadixBins = 1 << kRadixBits;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int logits_elem_bytes(int dtype) { return dtype == SIRLLM_F32 ? 4 : 2; }
+
+int validate_config(const sirllm_config* cfg);
+WorkspaceLayout workspace_layout(const sirllm_config& cfg);
+
+struct ScoreParams {
+    const void* logits;
+    const int32_t* token_ids;
+    const int32_t* n_new;  // nullable: max_new for every stream
+    float2* partials;
+    int64_t vocab;
+    int64_t row_stride;
+    int32_t n_streams, max_new, n_seg, logits_dtype;
+};
+
+struct SelectParams {
+    ScoreParams sc;        // used when score_new != 0
+    float* new_entropy;    // nullable
+    float* scores;
+    int64_t* serial;       // nullable
+    int32_t* live_len;
+    const float* decay;
+    int32_t* keep_idx;
+    int32_t* n_keep;
+    int32_t* first_moved;
+    int32_t* status;
+    int32_t capacity, budget, n_sink, n_recent, threshold;
+    int32_t compact_scores;  // also gather scores / serial and commit live_len
+    int32_t score_new;       // finish and append the scores of the round's new tokens first
+};
+
+struct CompactParams {
+    const char* src[2];  // K, V (nullable)
+    char* dst[2];
+    const int32_t* keep_idx;
+    const int32_t* n_keep;
+    const int32_t* first_moved;
+    int32_t* status;
+    int64_t planes_per_tensor;  // n_streams * n_layers * n_kv_heads
+    int32_t planes_per_stream;
+    int32_t capacity, keep_stride, row_bytes;
+    int32_t in_place;
+};
+
+cudaError_t launch_score_partials(const ScoreParams& p, cudaStream_t st);
+cudaError_t launch_score_finalize(const ScoreParams& p, float* out_entropy, int32_t* status,
+                                  cudaStream_t st);
+cudaError_t launch_select(const SelectParams& p, int n_streams, cudaStream_t st);
+cudaError_t launch_compact_plan(const CompactParams& p, int n_streams, int32_t* first_moved,
+                                cudaStream_t st);
+cudaError_t launch_compact(const CompactParams& p, cudaStream_t st);
+
+// ---- small device helpers ----------------------------------------------------------------
+#ifdef __CUDACC__
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr double kLn2 = 0.6931471805599453;
+constexpr float kNegHuge = -3.0e38f;  // "no element seen yet" for a running maximum
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Order-preserving map from fp32 bit patterns to unsigned integers: a larger key is a
+// larger score; negatives sort below non-negatives and -0 below +0.
+__device__ __forceinline__ uint32_t order_key(uint32_t bits) {
+    return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+}
+
+// Combine the per-segment (scaled max M, sum S) pairs of one logits row, where
+// sum_v exp(z_v) = S * 2^M, and return the token's entropy  ln(sum exp z) - z_id  (>= 0).
+__device__ __forceinline__ float finish_entropy(const float2* __restrict__ part, int n_seg,
+                                                float z_id) {
+    float M = kNegHuge;
+    for (int i = 0; i < n_seg; ++i) M = fmaxf(M, part[i].x);
+    double S = 0.0;
+    for (int i = 0; i < n_seg; ++i) S += (double)part[i].y * exp2((double)part[i].x - (double)M);
+    double e = ((double)M * kLn2 + log(S)) - (double)z_id;
+    return fmaxf((float)e, 0.0f);
+}
+
+__device__ __forceinline__ float load_logit(const void* logits, int dtype, int64_t idx) {
+    if (dtype == SIRLLM_F32) return ((const float*)logits)[idx];
+    return __uint_as_float((uint32_t)((const uint16_t*)logits)[idx] << 16);
+}
+#endif
+
+}  // namespace sirllm

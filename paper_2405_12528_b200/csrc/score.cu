@@ -1,0 +1,183 @@
+// Token Entropy (Section 3.2): e = -log softmax(z)[id] as a vocabulary-streaming
+// log-sum-exp.  Every logits row is cut into segments of kVecPerSeg 16-byte vectors;
+// one warp reduces one segment with an online (running-max) softmax sum and writes a
+// (scaled max, sum) pair.  The pairs of a row are combined in fp64 by whoever needs the
+// score: score_finalize_kernel here, or the selection kernel in the fused round.
+//
+// The kernel is bound by HBM reads (2 or 4 bytes per element, each read once); the
+// arithmetic per element is one conversion, one max, one FMA, one ex2 and one add.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace sirllm {
+
+namespace {
+
+constexpr int kUnroll = 4;  // 16-byte loads in flight per lane and loop trip
+
+__device__ __forceinline__ uint4 ld_stream_v4(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// Running state of one lane: sum_v 2^(z_v*log2e - mL), with mL = (max so far)*log2e
+// rounded once; the same rounded value is subtracted inside the FMA, so the pair
+// (mL, sum) represents sum_v exp(z_v) = sum * 2^mL without a systematic error.
+struct Online {
+    float mL = kNegHuge;
+    float s0 = 0.f, s1 = 0.f;
+    __device__ __forceinline__ void raise(float group_max) {
+        float cL = group_max * kLog2e;
+        if (cL > mL) {
+            float r = ex2_approx(mL - cL);
+            s0 *= r;
+            s1 *= r;
+            mL = cL;
+        }
+    }
+    __device__ __forceinline__ void add0(float z) { s0 += ex2_approx(fmaf(z, kLog2e, -mL)); }
+    __device__ __forceinline__ void add1(float z) { s1 += ex2_approx(fmaf(z, kLog2e, -mL)); }
+};
+
+__device__ __forceinline__ uint32_t bf162_max(uint32_t a, uint32_t b) {
+    __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&a);
+    __nv_bfloat162 y = *reinterpret_cast<__nv_bfloat162*>(&b);
+    __nv_bfloat162 m = __hmax2(x, y);
+    return *reinterpret_cast<uint32_t*>(&m);
+}
+
+template <bool kBf16>
+__global__ void __launch_bounds__(kScoreWarpsPerCta * 32)
+score_partials_kernel(const ScoreParams p) {
+    constexpr int ES = kBf16 ? 2 : 4;
+    constexpr int EPV = 16 / ES;
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * kScoreWarpsPerCta + (threadIdx.x >> 5);
+    const int64_t total = (int64_t)p.n_streams * p.max_new * p.n_seg;
+    if (warp >= total) return;
+    const int seg = (int)(warp % p.n_seg);
+    const int64_t row = warp / p.n_seg;
+    const int s = (int)(row / p.max_new);
+    const int t = (int)(row - (int64_t)s * p.max_new);
+    if (p.n_new != nullptr && t >= p.n_new[s]) return;
+
+    const int64_t V = p.vocab;
+    const char* rowp = (const char*)p.logits + row * p.row_stride * ES;
+    // elements in front of the first 16-byte boundary, whole vectors, elements after them
+    int64_t head = (int64_t)(((16u - (uint32_t)((uintptr_t)rowp & 15u)) & 15u) / ES);
+    if (head > V) head = V;
+    const int64_t nvec = (V - head) / EPV;
+    const int64_t tail = V - head - nvec * EPV;
+    const uint4* vec = (const uint4*)(rowp + head * ES);
+    const int64_t v0 = (int64_t)seg * kVecPerSeg;
+    const int64_t v1 = min(v0 + (int64_t)kVecPerSeg, nvec);
+    const uint32_t neg_inf = kBf16 ? 0xFF80FF80u : 0xFF800000u;
+
+    Online st;
+    for (int64_t base = v0; base < v1; base += 32 * kUnroll) {
+        uint4 x[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int64_t idx = base + u * 32 + lane;
+            if (idx < v1)
+                x[u] = ld_stream_v4(vec + idx);
+            else
+                x[u] = make_uint4(neg_inf, neg_inf, neg_inf, neg_inf);
+        }
+        if (kBf16) {
+            uint32_t m2 = x[0].x;
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                m2 = bf162_max(m2, x[u].x);
+                m2 = bf162_max(m2, x[u].y);
+                m2 = bf162_max(m2, x[u].z);
+                m2 = bf162_max(m2, x[u].w);
+            }
+            st.raise(fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u)));
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const uint32_t w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    st.add0(__uint_as_float(w[q] << 16));
+                    st.add1(__uint_as_float(w[q] & 0xFFFF0000u));
+                }
+            }
+        } else {
+            float gm = __uint_as_float(x[0].x);
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                gm = fmaxf(gm, fmaxf(fmaxf(__uint_as_float(x[u].x), __uint_as_float(x[u].y)),
+                                     fmaxf(__uint_as_float(x[u].z), __uint_as_float(x[u].w))));
+            }
+            st.raise(gm);
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                st.add0(__uint_as_float(x[u].x));
+                st.add1(__uint_as_float(x[u].y));
+                st.add0(__uint_as_float(x[u].z));
+                st.add1(__uint_as_float(x[u].w));
+            }
+        }
+    }
+    // ragged ends of the row (fewer than one vector each) go to segment 0
+    if (seg == 0 && lane < head + tail) {
+        const int64_t e = lane < head ? lane : head + nvec * EPV + (lane - head);
+        const float z = load_logit(rowp, kBf16 ? SIRLLM_BF16 : SIRLLM_F32, e);
+        st.raise(z);
+        st.add0(z);
+    }
+    // warp combine
+    float M = st.mL;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, o));
+    float S = (st.s0 + st.s1) * ex2_approx(st.mL - M);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(0xFFFFFFFFu, S, o);
+    if (lane == 0) p.partials[row * p.n_seg + seg] = make_float2(M, S);
+}
+
+__global__ void score_finalize_kernel(const ScoreParams p, float* __restrict__ out,
+                                      int32_t* __restrict__ status) {
+    const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= (int64_t)p.n_streams * p.max_new) return;
+    const int s = (int)(row / p.max_new);
+    const int t = (int)(row - (int64_t)s * p.max_new);
+    if (p.n_new != nullptr && t >= p.n_new[s]) return;
+    const int32_t id = p.token_ids[row];
+    float e = 0.f;
+    if (id >= 0 && (int64_t)id < p.vocab) {
+        const float z = load_logit(p.logits, p.logits_dtype, row * p.row_stride + id);
+        e = finish_entropy(p.partials + row * p.n_seg, p.n_seg, z);
+    } else if (id != -1) {
+        atomicOr(status, SIRLLM_STATUS_TOKEN_RANGE);
+    }
+    out[row] = e;
+}
+
+}  // namespace
+
+cudaError_t launch_score_partials(const ScoreParams& p, cudaStream_t st) {
+    const int64_t warps = (int64_t)p.n_streams * p.max_new * p.n_seg;
+    if (warps == 0) return cudaSuccess;
+    const unsigned grid = (unsigned)((warps + kScoreWarpsPerCta - 1) / kScoreWarpsPerCta);
+    if (p.logits_dtype == SIRLLM_BF16)
+        score_partials_kernel<true><<<grid, kScoreWarpsPerCta * 32, 0, st>>>(p);
+    else
+        score_partials_kernel<false><<<grid, kScoreWarpsPerCta * 32, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_score_finalize(const ScoreParams& p, float* out_entropy, int32_t* status,
+                                  cudaStream_t st) {
+    const int64_t rows = (int64_t)p.n_streams * p.max_new;
+    if (rows == 0) return cudaSuccess;
+    score_finalize_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, st>>>(p, out_entropy, status);
+    return cudaGetLastError();
+}
+
+}  // namespace sirllm

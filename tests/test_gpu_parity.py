@@ -1,0 +1,324 @@
+"""CUDA path against the CPU oracle, through the C ABI, on the same seeded inputs.
+
+Scores: within max(1e-5, 1e-4*|e|).  Keep lists, compacted scores, tags and K/V: bit exact
+(the oracle's selection consumes the GPU's scores, so both sides rank identical numbers).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import DeviceState, assert_entropy_close, oracle_twin
+from paper_2405_12528_b200 import binding as B
+from paper_2405_12528_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _score_cfg(T, V, dtype, stride=None, n_streams=1):
+    return B.make_config(n_streams, 1, 1, 8, 64, 16, 2, 2, T, V, dtype, torch.bfloat16,
+                         logits_row_stride=stride)
+
+
+# ------------------------------------------------------------------------------- scoring
+
+def test_score_tiny_workload_fp32():
+    w = wl.WORKLOADS["tiny"]
+    st = DeviceState(w, with_kv=False)
+    st.fill_round(0)
+    out = torch.full((w.new_tokens,), -1.0, device=DEV)
+    B.sirllm_score(st.cfg, st.logits, st.token_ids, None, out, st.ws)
+    want = oracle.score(st.logits.cpu(), st.token_ids.cpu())
+    assert_entropy_close(out, want)
+    assert B.sirllm_status(st.ws) == 0
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("V,stride", [(1, None), (2, None), (7, 9), (33, None), (4095, 4099),
+                                      (4096, None), (8193, 8200), (32000, None), (50257, 50257)])
+def test_score_ragged_vocabularies_and_strides(dtype, V, stride):
+    # odd V and odd strides put rows off the 16-byte grid: ragged head and tail per row;
+    # V > 4096 (bf16) / 2048 (fp32) spans several segments
+    T = 19
+    stride = V if stride is None else stride
+    g = torch.Generator().manual_seed(V)
+    buf = (torch.randn(T, stride, generator=g) * 3).to(dtype)
+    ids = torch.randint(0, V, (T,), generator=g, dtype=torch.int32)
+    cfg = _score_cfg(T, V, dtype, stride)
+    ws = B.new_workspace(cfg)
+    out = torch.zeros(T, device=DEV)
+    d_buf = buf.to(DEV)
+    B.sirllm_score(cfg, d_buf[:, :V] if stride != V else d_buf, ids.to(DEV), None, out, ws)
+    assert_entropy_close(out, oracle.score(buf[:, :V], ids))
+
+
+def test_score_closed_forms_on_device():
+    import math
+    V = 32000
+    cfg = _score_cfg(3, V, torch.float32)
+    ws = B.new_workspace(cfg)
+    z = torch.zeros(3, V)
+    z[1, 77] = 80.0
+    z[2] = -5.0
+    z[2, 0] = float("-inf")              # a masked column
+    ids = torch.tensor([5, 77, 9], dtype=torch.int32)
+    out = torch.zeros(3, device=DEV)
+    B.sirllm_score(cfg, z.to(DEV), ids.to(DEV), None, out, ws)
+    out = out.cpu()
+    assert abs(float(out[0]) - math.log(V)) < 1e-5
+    assert float(out[1]) == 0.0
+    assert abs(float(out[2]) - math.log(V - 1)) < 1e-5
+
+
+def test_score_special_ids_ragged_streams_and_status():
+    S, M, V = 3, 8, 1000
+    cfg = _score_cfg(M, V, torch.bfloat16, n_streams=S)
+    ws = B.new_workspace(cfg)
+    g = torch.Generator().manual_seed(0)
+    logits = (torch.randn(S * M, V, generator=g) * 2).to(torch.bfloat16)
+    ids = torch.randint(0, V, (S * M,), generator=g, dtype=torch.int32)
+    ids[0], ids[9], ids[10] = -1, V, -5
+    n_new = torch.tensor([8, 3, 0], dtype=torch.int32)
+    out = torch.full((S * M,), -7.0, device=DEV)
+    B.sirllm_score(cfg, logits.to(DEV), ids.to(DEV), n_new.to(DEV), out, ws)
+    out = out.cpu()
+    want = oracle.score(logits, ids)
+    live = torch.zeros(S * M, dtype=torch.bool)
+    for s in range(S):
+        live[s * M:s * M + int(n_new[s])] = True
+    assert_entropy_close(out[live], want[live])
+    assert (out[~live] == -7.0).all()                    # rows beyond n_new are not touched
+    assert out[0] == 0.0 and out[9] == 0.0 and out[10] == 0.0
+    assert B.sirllm_status(ws, clear=True) == B.STATUS_TOKEN_RANGE
+    assert B.sirllm_status(ws) == 0
+
+
+# ------------------------------------------------------------------------------- selection
+
+def _select_case(l_list, n_sink, n_recent, budget, threshold, cap, seed, quantise, decay, compact):
+    S = len(l_list)
+    cfg = B.make_config(S, 1, 1, 8, cap, budget, n_sink, n_recent, 0, 16, torch.float32,
+                        torch.bfloat16, threshold=threshold)
+    ws = B.new_workspace(cfg)
+    E = torch.zeros(S, cap)
+    serial = torch.full((S, cap), -1, dtype=torch.int64)
+    for s, l in enumerate(l_list):
+        E[s, :l] = wl.random_scores(seed + s, l, quantise=quantise)
+        serial[s, :l] = torch.arange(l) * 3 + s
+    dE, dser = E.to(DEV), serial.to(DEV)
+    dlen = torch.tensor(l_list, dtype=torch.int32, device=DEV)
+    ddec = torch.tensor(decay, dtype=torch.float32, device=DEV)
+    keep = torch.full((S, threshold), -1, dtype=torch.int32, device=DEV)
+    nk = torch.zeros(S, dtype=torch.int32, device=DEV)
+    B.sirllm_decay_select(cfg, dE, dser, dlen, ddec, keep, nk, compact, ws)
+    assert B.sirllm_status(ws) == 0
+    for s, l in enumerate(l_list):
+        Es = E[s].clone()
+        oracle.decay(Es, l, decay[s])
+        want = oracle.select(Es, l, n_sink, n_recent, budget, threshold)
+        n = int(nk[s])
+        assert n == len(want)
+        assert torch.equal(keep[s, :n].cpu(), want)
+        if compact:
+            assert int(dlen[s]) == n
+            assert torch.equal(dE[s, :n].cpu().view(torch.int32), Es[want.long()].view(torch.int32))
+            assert torch.equal(dser[s, :n].cpu(), serial[s][want.long()])
+        else:
+            assert int(dlen[s]) == l
+            assert torch.equal(dE[s, :l].cpu().view(torch.int32), Es[:l].view(torch.int32))
+            assert torch.equal(dser[s].cpu(), serial[s])
+
+
+@pytest.mark.parametrize("compact", [False, True])
+@pytest.mark.parametrize("quantise", [0, 5])
+def test_select_matches_oracle(compact, quantise):
+    _select_case([5000, 3000, 2049, 2048, 100, 0], 4, 256, 2048, 2048, 5120, 1, quantise,
+                 [0.9, 0.5, 1.0, 0.7, 0.8, 0.9], compact)
+
+
+def test_select_paper_shaped_rows_no_recent_window():
+    # Tables 1-3: 4 sinks + 508 (1020) entropy slots, no recent window
+    _select_case([632, 513], 4, 0, 512, 512, 640, 3, 0, [0.7, 0.5], True)
+    _select_case([1078], 4, 0, 1024, 1024, 1152, 4, 7, [0.8], True)
+
+
+def test_select_degenerate_shapes():
+    _select_case([300], 4, 28, 32, 32, 512, 5, 0, [0.9], True)       # k = 0: StreamLLM
+    _select_case([300], 0, 32, 32, 32, 512, 6, 0, [0.9], True)       # sliding window
+    _select_case([300], 0, 0, 32, 32, 512, 7, 3, [0.9], True)        # pure top-k with ties
+    _select_case([300, 41], 4, 4, 40, 200, 512, 8, 0, [0.9, 0.9], True)   # threshold > budget
+    _select_case([33], 4, 4, 32, 32, 64, 9, 2, [1.0], True)          # evict exactly one
+
+
+def test_select_largest_capacity_and_all_equal_scores():
+    cap = B.MAX_CAPACITY
+    _select_case([cap], 4, 1024, 8192, 8192, cap, 10, 0, [0.9], True)
+    S, l = 1, 4000
+    cfg = B.make_config(S, 1, 1, 8, 4096, 1000, 4, 96, 0, 16, torch.float32, torch.bfloat16)
+    ws = B.new_workspace(cfg)
+    E = torch.full((1, 4096), 2.5, device=DEV)
+    keep = torch.zeros(1, 1000, dtype=torch.int32, device=DEV)
+    nk = torch.zeros(1, dtype=torch.int32, device=DEV)
+    dlen = torch.tensor([l], dtype=torch.int32, device=DEV)
+    B.sirllm_decay_select(cfg, E, None, dlen, torch.tensor([0.5], device=DEV), keep, nk, 0, ws)
+    assert keep[0].cpu().tolist() == list(range(904)) + list(range(l - 96, l))
+
+
+def test_select_special_values_follow_the_bit_pattern_order():
+    vals = torch.tensor([0.0, -0.0, 1e-45, -1e-45, float("inf"), -float("inf"), 1.0, -1.0,
+                         1.17549435e-38, 3.0, 3.0, 2.0, 0.0, -0.0, 5e-324, 7.0])
+    l = vals.numel()
+    cfg = B.make_config(1, 1, 1, 8, 32, 6, 0, 0, 0, 16, torch.float32, torch.bfloat16)
+    ws = B.new_workspace(cfg)
+    E = torch.zeros(1, 32)
+    E[0, :l] = vals
+    dE = E.to(DEV)
+    keep = torch.zeros(1, 6, dtype=torch.int32, device=DEV)
+    nk = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for budget in (6, 11, 13):
+        cfg = B.make_config(1, 1, 1, 8, 32, budget, 0, 0, 0, 16, torch.float32, torch.bfloat16)
+        keep = torch.zeros(1, budget, dtype=torch.int32, device=DEV)
+        d = E.to(DEV)
+        B.sirllm_decay_select(cfg, d, None, torch.tensor([l], dtype=torch.int32, device=DEV),
+                              torch.tensor([1.0], device=DEV), keep, nk, 0, ws)
+        want = oracle.select(E[0].clone(), l, 0, 0, budget)
+        assert torch.equal(keep[0].cpu(), want)
+
+
+# ------------------------------------------------------------------------------- compaction
+
+def _compact_case(S, planes, cap, D, n_list, in_place, seed, dtype=torch.bfloat16):
+    thr = max(n_list + [1])
+    cfg = B.make_config(S, planes, 1, D, cap, thr, 0, 0, 0, 16, torch.float32, dtype)
+    ws = B.new_workspace(cfg)
+    g = torch.Generator().manual_seed(seed)
+    k = torch.randn(S, planes, cap, D, generator=g).to(dtype)
+    v = torch.randn(S, planes, cap, D, generator=g).to(dtype)
+    keep = torch.full((S, thr), -1, dtype=torch.int32)
+    for s, n in enumerate(n_list):
+        keep[s, :n] = torch.sort(torch.randperm(cap, generator=g)[:n]).values.to(torch.int32)
+    dk, dv = k.to(DEV), v.to(DEV)
+    dkeep, dn = keep.to(DEV), torch.tensor(n_list, dtype=torch.int32, device=DEV)
+    if in_place:
+        B.sirllm_compact_kv(cfg, dk, dv, dk, dv, dkeep, dn, ws)
+        ok, ov = dk, dv
+    else:
+        ok = torch.full_like(dk, 9.0)
+        ov = torch.full_like(dv, 9.0)
+        B.sirllm_compact_kv(cfg, dk, dv, ok, ov, dkeep, dn, ws)
+        assert torch.equal(dk.cpu(), k) and torch.equal(dv.cpu(), v)      # sources untouched
+    assert B.sirllm_status(ws) == 0
+    ok, ov = ok.cpu(), ov.cpu()
+    for s, n in enumerate(n_list):
+        for p in range(planes):
+            assert torch.equal(ok[s, p, :n], oracle.gather_rows(k[s, p], keep[s, :n]))
+            assert torch.equal(ov[s, p, :n], oracle.gather_rows(v[s, p], keep[s, :n]))
+            if not in_place:
+                assert (ok[s, p, n:] == 9.0).all()                        # nothing written past n_keep
+            else:
+                # slots never used as a destination keep their old rows
+                assert torch.equal(ok[s, p, n:], k[s, p, n:])
+
+
+@pytest.mark.parametrize("in_place", [True, False])
+def test_compact_matches_gather(in_place):
+    _compact_case(2, 5, 300, 128, [200, 37], in_place, 0)
+    _compact_case(1, 3, 1000, 64, [999], in_place, 1, torch.float16)       # ragged last chunk
+    _compact_case(3, 2, 64, 8, [0, 1, 64], in_place, 2)                    # empty, single, full
+    _compact_case(1, 700, 96, 128, [50], in_place, 3)                      # more planes than workers
+
+
+def test_compact_identity_list_moves_nothing_and_bad_lists_are_refused():
+    cfg = B.make_config(2, 2, 1, 16, 40, 20, 0, 0, 0, 16, torch.float32, torch.bfloat16)
+    ws = B.new_workspace(cfg)
+    k = torch.randn(2, 2, 40, 16).to(torch.bfloat16)
+    dk = k.to(DEV)
+    keep = torch.stack([torch.arange(20), torch.arange(20)]).to(torch.int32)
+    keep[1, 5], keep[1, 6] = 9, 8                              # not ascending
+    n = torch.tensor([20, 20], dtype=torch.int32, device=DEV)
+    B.sirllm_compact_kv(cfg, dk, None, dk, None, keep.to(DEV), n, ws)
+    assert B.sirllm_status(ws, clear=True) == B.STATUS_BAD_KEEP
+    assert torch.equal(dk.cpu(), k)
+    keep[1] = torch.arange(20) + 30                            # runs past the capacity
+    B.sirllm_compact_kv(cfg, dk, None, dk, None, keep.to(DEV), n, ws)
+    assert B.sirllm_status(ws, clear=True) == B.STATUS_BAD_KEEP
+    assert torch.equal(dk.cpu(), k)
+
+
+# ------------------------------------------------------------------------------- whole rounds
+
+def _run_stream(w, rounds, ragged=False, seed=0, check_kv_host=True, rho=None):
+    st = DeviceState(w, seed=seed)
+    twins = oracle_twin(w, st.decay.cpu())
+    M = st.cfg.max_new
+    for r in range(rounds):
+        n_new = None
+        if ragged:
+            n_new = wl.ragged_lengths(seed, w.n_streams, r, w.new_tokens).tolist()
+        n_new = st.fill_round(r, n_new, rho)
+        # GPU scores first (the same kernel the fused round runs), for the oracle to rank
+        e_gpu = torch.zeros_like(st.new_entropy)
+        B.sirllm_score(st.cfg, st.logits, st.token_ids, st.n_new, e_gpu, st.ws)
+        before = [t.live_len for t in twins]
+        st.step()
+        assert B.sirllm_status(st.ws) == 0
+        e_gpu = e_gpu.cpu()
+        for s, tw in enumerate(twins):
+            T, l = n_new[s], before[s]
+            rows = slice(s * M, s * M + T)
+            want_e = oracle.score(st.logits[rows].cpu(), st.token_ids[rows].cpu())
+            assert_entropy_close(e_gpu[rows], want_e)                          # P1
+            assert torch.equal(st.new_entropy[rows].cpu().view(torch.int32),
+                               e_gpu[rows].view(torch.int32))                  # fused == standalone
+            serials = torch.arange(int(tw.next_serial.value), int(tw.next_serial.value) + T)
+            tw.k[:, l:l + T] = wl.make_kv_rows(w, seed, "k", s, serials)
+            tw.v[:, l:l + T] = wl.make_kv_rows(w, seed, "v", s, serials)
+            keep = tw.step(e_gpu[rows])                                        # P2: same scores
+            n = tw.live_len
+            assert st.host_len[s] == n and int(st.n_keep[s]) == n
+            assert torch.equal(st.keep_idx[s, :n].cpu(), keep)
+            assert torch.equal(st.scores[s, :n].cpu().view(torch.int32), tw.E[:n].view(torch.int32))
+            assert torch.equal(st.serial[s, :n].cpu(), tw.serial[:n])
+            if check_kv_host:                                                  # P3
+                assert torch.equal(st.k[s, :, :n].cpu(), tw.k[:, :n])
+                assert torch.equal(st.v[s, :, :n].cpu(), tw.v[:, :n])
+        st.check_kv_by_content()
+    return st
+
+
+def test_step_tiny_workload():
+    st = _run_stream(wl.WORKLOADS["tiny"], 1)
+    assert st.host_len == [256]
+
+
+def test_step_multi_round_small_stream():
+    w = wl.WORKLOADS["mistral_7b_gqa"].scaled(n_layers=2, n_kv_heads=3, capacity=1536, budget=1024,
+                                              n_recent=128, new_tokens=200, vocab=5003)
+    _run_stream(w, 12)
+
+
+def test_step_ragged_multi_stream_rounds():
+    w = wl.WORKLOADS["batched64"].scaled(n_streams=5, n_layers=2, n_kv_heads=2, capacity=512,
+                                         budget=256, n_recent=64, new_tokens=100, vocab=4099)
+    _run_stream(w, 10, ragged=True)
+
+
+def test_step_paper_shaped_small_rounds():
+    w = wl.WORKLOADS["rps_1024"].scaled(n_layers=2, n_kv_heads=2, vocab=32000)
+    _run_stream(w, 30, rho=0.0)
+
+
+def test_step_overflowing_round_is_skipped_and_flagged():
+    w = wl.WORKLOADS["tiny"].scaled(n_streams=2, n_layers=1, n_kv_heads=1, capacity=300, budget=256,
+                                    new_tokens=200, vocab=1000)
+    st = DeviceState(w, threshold=300)            # no eviction below 300: the 2nd round cannot fit
+    st.fill_round(0)
+    st.step()
+    assert st.host_len == [200, 200]
+    snap = (st.scores.clone(), st.k.clone(), st.serial.clone())
+    st.fill_round(1, [200, 50])
+    st.step()
+    assert B.sirllm_status(st.ws, clear=True) == B.STATUS_OVERFLOW
+    assert st.host_len == [200, 250]
+    assert torch.equal(st.scores[0], snap[0][0]) and torch.equal(st.k[0], snap[1][0])
