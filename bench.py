@@ -1,0 +1,448 @@
+#!/usr/bin/env python
+"""Throughput of the SirLLM retention pass (score -> append -> decay -> select -> compact).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A step is one evicting round of the whole pass over one batch of synthetic input at steady
+state (live length = budget before the round's tokens arrive).  One JSON line is printed by
+rank 0.  Under torchrun every rank drives its own GPU with its own independent streams (the
+pass shards by stream; there is no collective on the data path) and the line reports the
+whole job: weak scaling.
+
+Timing: CUDA events on the launching stream, barrier + synchronize on both sides, max over
+ranks.  The K timed rounds run back to back; every round reads a logits tensor (>= 1 GB on
+the default workload) and a K/V cache (>= 2 GB) far larger than the 126 MB L2, and
+alternates between two logits tensors, so nothing it needs is cache resident.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2405_12528_b200 import workloads as wl  # noqa: E402
+
+METRIC = "tokens/s through entropy+decay+top-k eviction; KV compaction GB/s vs HBM peak"
+UNIT = "tokens/s"
+DEFAULT_WORKLOAD = "llama3_8b"      # the shape the 70 %-of-HBM target is quoted on
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_hbm_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while a region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc = index, None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        self.result = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            return
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            self.result = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx),
+                           "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------
+# the CUDA arm
+# --------------------------------------------------------------------------------------------
+
+class Pass:
+    """Device state of one rank and the calls of one round."""
+
+    def __init__(self, w: wl.Workload, seed: int, dev: str):
+        from paper_2405_12528_b200 import binding as B
+        self.B, self.w, self.seed, self.dev = B, w, seed, dev
+        self.cfg = B.config_from_workload(w)
+        S, P, C, D, M = w.n_streams, w.planes_per_stream, w.capacity, w.head_dim, w.new_tokens
+        self.ws = B.new_workspace(self.cfg, dev)
+        self.scores = torch.zeros(S, C, dtype=torch.float32, device=dev)
+        self.serial = torch.full((S, C), -1, dtype=torch.int64, device=dev)
+        self.live_len = torch.zeros(S, dtype=torch.int32, device=dev)
+        self.decay = wl.stream_decay(w, seed).to(dev)
+        self.keep_idx = torch.zeros(S, self.cfg.threshold, dtype=torch.int32, device=dev)
+        self.n_keep = torch.zeros(S, dtype=torch.int32, device=dev)
+        self.new_entropy = torch.zeros(S * M, dtype=torch.float32, device=dev)
+        self.k = torch.zeros(S, P, C, D, dtype=w.torch_kv_dtype, device=dev)
+        self.v = torch.zeros(S, P, C, D, dtype=w.torch_kv_dtype, device=dev)
+        self.n_new = torch.full((S,), M, dtype=torch.int32, device=dev)
+        bias = wl.zipf_bias_table(w.vocab, w.zipf_bias, dev) if w.zipf_bias else None
+        self.pool = []                    # two rounds of logits / ids to alternate between
+        for r in range(2):
+            lg = torch.empty(S * M, w.vocab, dtype=w.torch_logits_dtype, device=dev)
+            ids = torch.empty(S * M, dtype=torch.int32, device=dev)
+            for s in range(S):
+                wl.make_logits(w, seed, s, r, M, dev, bias, out=lg[s * M:(s + 1) * M])
+                ids[s * M:(s + 1) * M] = wl.make_token_ids(w, seed, s, r, M, dev)
+            self.pool.append((lg, ids))
+        self.next_serial = 0
+        self.round = 0
+
+    def append_rows(self):
+        """Stand-in for the model: writes the round's new K/V rows and tags behind the live rows."""
+        w = self.w
+        lens = self.live_len.cpu().tolist()
+        T = w.new_tokens
+        serials = torch.arange(self.next_serial, self.next_serial + T, device=self.dev)
+        for s in range(w.n_streams):
+            l = lens[s]
+            self.serial[s, l:l + T] = serials
+            self.k[s, :, l:l + T] = wl.make_kv_rows(w, self.seed, "k", s, serials, device=self.dev)
+            self.v[s, :, l:l + T] = wl.make_kv_rows(w, self.seed, "v", s, serials, device=self.dev)
+        self.next_serial += T
+
+    def step(self, events=None):
+        lg, ids = self.pool[self.round & 1]
+        self.round += 1
+        args = (self.cfg, lg, ids, self.n_new, self.scores, self.serial, self.live_len, self.decay,
+                self.k, self.v, self.keep_idx, self.n_keep, self.new_entropy, self.ws)
+        if events is None:
+            self.B.sirllm_step(*args)
+        else:
+            self.B.sirllm_step_phases(*args, events)
+
+    def prime(self):
+        """Real rounds from an empty cache until the first eviction has happened."""
+        w = self.w
+        n = (w.budget + w.new_tokens - 1) // w.new_tokens + 1
+        for _ in range(n):
+            self.append_rows()
+            self.step()
+        assert self.live_len.cpu().tolist() == [w.budget] * w.n_streams
+        assert self.B.sirllm_status(self.ws) == 0
+
+    def moved_rows(self):
+        """Rows that changed slot in the last round, summed over streams (in-place traffic)."""
+        j = torch.arange(self.cfg.threshold, device=self.dev, dtype=torch.int32)
+        moved = (self.keep_idx != j[None, :]) & (j[None, :] < self.n_keep[:, None])
+        return int(moved.sum())
+
+
+def step_bytes(w: wl.Workload, moved_rows: int) -> dict:
+    """Algorithmic bytes of one round: logits read once (+ ids, target logit sector, score
+    written), scores read+written, keep list; every moved K/V row read once and written once."""
+    es = 4 if w.logits_dtype == "f32" else 2
+    T = w.n_streams * w.new_tokens
+    l = w.n_streams * (w.budget + w.new_tokens)
+    score = T * w.vocab * es + T * (4 + 32 + 4)
+    select = 2 * l * 4 + w.n_streams * w.budget * 4
+    compact = 2 * moved_rows * w.row_bytes * 2 * w.planes_per_stream
+    return {"score": score, "select": select, "compact": compact, "step": score + select + compact}
+
+
+def run_ours(args, rank, world, local_rank):
+    from paper_2405_12528_b200 import binding as B
+    B.lib()                                       # fail loudly if the CUDA library is missing
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    w = wl.WORKLOADS[args.workload]
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    p = Pass(w, seed=rank, dev=dev)
+    p.prime()
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = oracle_rounds(p, rounds=3)
+
+    def sync():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        p.step()
+    sync()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clk:
+        t0.record()
+        for _ in range(args.steps):
+            p.step()
+        t1.record()
+        sync()
+    ms_total = t0.elapsed_time(t1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t[0])
+    assert B.sirllm_status(p.ws) == 0
+    ms_step = ms_total / args.steps
+    tokens = world * w.n_streams * w.new_tokens
+    value = tokens / (ms_step * 1e-3)
+
+    # per-phase durations of the same rounds (events between the three launches)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    phase_ms, moved = [0.0, 0.0, 0.0], []
+    for i in range(args.steps):
+        p.step(evs[i])
+        torch.cuda.synchronize()
+        moved.append(p.moved_rows())
+        for j in range(3):
+            phase_ms[j] += evs[i][j].elapsed_time(evs[i][j + 1]) / args.steps
+    peak, peak_kind = measured_hbm_peak()
+    mean_moved = sum(moved) / len(moved)
+    by = step_bytes(w, mean_moved)
+    compact_gbs = by["compact"] / (phase_ms[2] * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "compact_kernel", "achieved": round(compact_gbs, 1),
+                "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": round(compact_gbs / peak, 4), "traffic": None,
+                "bytes_per_launch": by["compact"], "ms_per_launch": round(phase_ms[2], 4),
+                "moved_rows_per_round": mean_moved,
+                "phases_ms": {"score": round(phase_ms[0], 4), "select": round(phase_ms[1], 4),
+                              "compact": round(phase_ms[2], 4)},
+                "score_gbs": round(by["score"] / (phase_ms[0] * 1e-3) / 1e9, 1),
+                "step_bytes": by["step"],
+                "step_gbs": round(by["step"] / (ms_step * 1e-3) / 1e9, 1),
+                "step_frac": round(by["step"] / (ms_step * 1e-3) / 1e9 / peak, 4),
+                "step_frac_of_8000": round(by["step"] / (ms_step * 1e-3) / 1e9 / 8000.0, 4)}
+
+    e2e = run_e2e(p, args, dist, world)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_step, 4),
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32", "data": "synthetic",
+                "config": {"workload": w.name, "streams_per_gpu": w.n_streams,
+                           "new_tokens_per_round": w.new_tokens, "vocab": w.vocab,
+                           "logits_dtype": w.logits_dtype, "kv_dtype": w.kv_dtype,
+                           "planes": 2 * w.planes_per_stream, "head_dim": w.head_dim,
+                           "capacity": w.capacity, "budget": w.budget, "n_sink": w.n_sink,
+                           "n_recent": w.n_recent, "decay": w.decay, "parallelism": f"streams x{world}",
+                           "l2": "inputs larger than L2 (logits alternate between two tensors)"},
+                "clocks": clk.result, "e2e": e2e, "gpu_launches": 3 * args.steps,
+                "roofline": roofline}
+        if cpu_baseline is not None:
+            line["cpu_baseline"] = cpu_baseline
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_e2e(p: Pass, args, dist, world):
+    """The same rounds through sirllm_step_host: inputs start in pinned host memory, the
+    round's results (keep lists, new lengths, new scores) end in pinned host memory."""
+    w, B, cfg = p.w, p.B, p.cfg
+    S, P, M, D = w.n_streams, w.planes_per_stream, w.new_tokens, w.head_dim
+    pin = lambda t: t.cpu().pin_memory()
+    h_pool = [(pin(lg), pin(ids)) for lg, ids in p.pool]
+    serials = torch.arange(M, device=p.dev)
+    h_k = torch.empty(S, P, M, D, dtype=w.torch_kv_dtype).pin_memory()
+    h_v = torch.empty(S, P, M, D, dtype=w.torch_kv_dtype).pin_memory()
+    for s in range(S):
+        h_k[s] = wl.make_kv_rows(w, p.seed, "k", s, serials, device=p.dev).cpu()
+        h_v[s] = wl.make_kv_rows(w, p.seed, "v", s, serials, device=p.dev).cpu()
+    h_n_new = torch.full((S,), M, dtype=torch.int32).pin_memory()
+    h_len = p.live_len.cpu().pin_memory()
+    h_keep = torch.zeros(S, cfg.threshold, dtype=torch.int32).pin_memory()
+    h_nk = torch.zeros(S, dtype=torch.int32).pin_memory()
+    h_e = torch.zeros(S * M, dtype=torch.float32).pin_memory()
+    d_logits, d_ids = p.pool[0]
+    h2d = sum(t.numel() * t.element_size() for t in (h_pool[0][0], h_pool[0][1], h_k, h_v, h_n_new))
+    d2h = sum(t.numel() * t.element_size() for t in (h_keep, h_nk, h_e))
+
+    def one(i):
+        lg, ids = h_pool[i & 1]
+        B.sirllm_step_host(cfg, lg, ids, h_n_new, h_k, h_v, h_len, d_logits, d_ids, p.n_new,
+                           p.scores, p.serial, p.live_len, p.decay, p.k, p.v, p.keep_idx, p.n_keep,
+                           p.new_entropy, h_keep, h_nk, h_e, p.ws)
+        torch.cuda.current_stream().synchronize()      # the caller reads the results
+        h_len.copy_(h_nk)
+
+    n = max(2, min(args.steps, 10))
+    for i in range(2):
+        one(i)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for i in range(n):
+        one(i)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([dt], device=p.dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = float(t[0])
+    return {"value": round(world * S * M * n / dt, 1), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": round(dt / n * 1e3, 3), "steps": n,
+            "call": "sirllm_step_host"}
+
+
+# --------------------------------------------------------------------------------------------
+# the oracle on the host cores: CPU baseline of the CUDA arm and the reference arm
+# --------------------------------------------------------------------------------------------
+
+def oracle_rounds(p: Pass, rounds: int):
+    """Times `rounds` full evicting rounds of the oracle, as it stands, on a host copy of the
+    device state (1 thread)."""
+    import oracle
+    w = p.w
+    S, M = w.n_streams, w.new_tokens
+    p.append_rows()
+    torch.cuda.synchronize()
+    lg, ids = p.pool[0]
+    h_lg, h_ids = lg.cpu(), ids.cpu()
+    streams = []
+    for s in range(S):
+        st = oracle.Stream(w.capacity, w.n_sink, w.n_recent, w.budget, w.threshold, float(p.decay[s]),
+                           p.k[s].cpu(), p.v[s].cpu())
+        st.E.copy_(p.scores[s].cpu())
+        st.live_len = int(p.live_len[s])
+        streams.append(st)
+    t0 = time.perf_counter()
+    for _ in range(rounds):
+        for s, st in enumerate(streams):
+            e = oracle.score(h_lg[s * M:(s + 1) * M], h_ids[s * M:(s + 1) * M])
+            st.step(e)
+    dt = time.perf_counter() - t0
+    return {"value": round(rounds * S * M / dt, 1), "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{rounds} full evicting rounds of {w.name} (all {S * M} tokens, all "
+                      f"{2 * w.planes_per_stream * S} planes), {dt:.1f} s of CPU time",
+            "seconds_per_round": round(dt / rounds, 3)}
+
+
+def run_reference(args, rank, world):
+    """The oracle, as it stands, on the host cores: the same workload, metric and unit."""
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    w = wl.WORKLOADS[args.workload]
+    # a bounded slice of the round: a fraction f of the new tokens and of the K/V planes
+    # (the pass is linear in both), so that K + W steps end within a few minutes
+    full_round_s = (w.n_streams * w.new_tokens * w.vocab / 1.4e8
+                    + 4 * w.n_streams * w.planes_per_stream * w.budget * w.row_bytes / 2.0e9)
+    f = 1.0
+    while f > 1 / 64 and full_round_s * f * (args.steps + args.warmup) > 120.0:
+        f /= 2
+    if w.n_streams > 1:      # whole streams first, then a slice of each
+        S = max(1, int(w.n_streams * f))
+        f = min(1.0, f * w.n_streams / S)
+    else:
+        S = 1
+    T = max(1, int(w.new_tokens * f))
+    P = max(1, int(w.planes_per_stream * f))
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    bias = wl.zipf_bias_table(w.vocab, w.zipf_bias, dev) if w.zipf_bias else None
+    planes = torch.arange(P)
+    streams, inputs = [], []
+    for s in range(S):
+        k = torch.zeros(P, w.capacity, w.head_dim, dtype=w.torch_kv_dtype)
+        v = torch.zeros_like(k)
+        st = oracle.Stream(w.capacity, w.n_sink, w.n_recent, w.budget, w.threshold,
+                           float(wl.stream_decay(w, 0)[s]), k, v)
+        first = torch.arange(w.budget)
+        k[:, :w.budget] = wl.make_kv_rows(w, 0, "k", s, first, planes, dev).cpu()
+        v[:, :w.budget] = wl.make_kv_rows(w, 0, "v", s, first, planes, dev).cpu()
+        st.E[:w.budget] = wl.random_scores(s, w.budget)
+        st.live_len = w.budget
+        st.next_serial.value = w.budget
+        streams.append(st)
+        inputs.append((wl.make_logits(w, 0, s, 0, T, dev, bias).cpu(),
+                       wl.make_token_ids(w, 0, s, 0, T, dev).cpu()))
+
+    def one():
+        for st, (lg, ids) in zip(streams, inputs):
+            e = oracle.score(lg, ids)
+            pad = torch.zeros(w.new_tokens - T)      # the rest of the round's tokens: score 0
+            st.step(torch.cat([e, pad]))
+
+    for _ in range(args.warmup):
+        one()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = S * T / dt
+    sample = (f"per step: {S} of {w.n_streams} streams, {T} of {w.new_tokens} new tokens scored and "
+              f"{2 * P} of {2 * w.planes_per_stream} K/V planes compacted per stream (the same "
+              f"fraction of both; selection over the full cache)")
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 1), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name},
+            "cpu_baseline": {"value": round(value, 1), "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": round(value, 1), "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

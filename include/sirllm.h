@@ -164,6 +164,31 @@ int sirllm_step_phases(const sirllm_config *cfg, const void *logits, const int32
                        const float *decay, void *k, void *v, int32_t *keep_idx, int32_t *n_keep,
                        float *new_entropy, void *ws, void *cuda_stream, void **phase_events);
 
+/*
+ * One whole round for a caller whose model outputs live in HOST memory (Algorithm 1's
+ * loop body, as sirllm_step): copies the round's inputs to the device, runs
+ * sirllm_step on them and copies the round's results back, all enqueued on the stream;
+ * the host outputs are valid once the stream has been synchronised.  Pinned host
+ * buffers let the copies run asynchronously.
+ *   (host) h_logits, h_token_ids  laid out as the device arrays of sirllm_step
+ *   (host) h_n_new  int32 [n_streams];  h_live_len int32 [n_streams]: the caller's copy
+ *          of the current live lengths (it tells where the new K/V rows go)
+ *   (host) h_new_k, h_new_v  [n_streams][planes][max_new][head_dim] the round's new rows,
+ *          or NULL when the rows are already in the device caches
+ *   d_logits, d_token_ids, d_n_new  device staging with the shapes sirllm_step expects
+ *   scores ... new_entropy          device state and outputs exactly as in sirllm_step,
+ *                                   keep_idx / n_keep / new_entropy required
+ *   (host) h_keep_idx [n_streams][threshold], h_n_keep [n_streams],
+ *          h_new_entropy [n_streams*max_new]  results (h_n_keep = the new live lengths)
+ */
+int sirllm_step_host(const sirllm_config *cfg, const void *h_logits, const int32_t *h_token_ids,
+                     const int32_t *h_n_new, const void *h_new_k, const void *h_new_v,
+                     const int32_t *h_live_len, void *d_logits, int32_t *d_token_ids,
+                     int32_t *d_n_new, float *scores, int64_t *serial, int32_t *live_len,
+                     const float *decay, void *k, void *v, int32_t *keep_idx, int32_t *n_keep,
+                     float *new_entropy, int32_t *h_keep_idx, int32_t *h_n_keep,
+                     float *h_new_entropy, void *ws, void *cuda_stream);
+
 /* Waits for the stream, copies the status word to *status_out (host) and, if
  * `clear` != 0, resets it.  No counterpart in the paper. */
 int sirllm_status(void *ws, void *cuda_stream, int32_t *status_out, int32_t clear);

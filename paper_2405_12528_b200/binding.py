@@ -22,7 +22,8 @@ STATUS_TOKEN_RANGE, STATUS_OVERFLOW, STATUS_TIMEOUT, STATUS_BAD_KEEP = 1, 2, 4, 
 MAX_CAPACITY = 49152
 
 EXPORTS = ["sirllm_workspace_bytes", "sirllm_workspace_init", "sirllm_score", "sirllm_decay_select",
-           "sirllm_compact_kv", "sirllm_step", "sirllm_step_phases", "sirllm_status", "sirllm_strerror",
+           "sirllm_compact_kv", "sirllm_step", "sirllm_step_phases", "sirllm_step_host",
+           "sirllm_status", "sirllm_strerror",
            "sirllm_last_cuda_error"]
 
 _DTYPE_CODE = {torch.float32: F32, torch.bfloat16: BF16, torch.float16: F16}
@@ -92,6 +93,8 @@ def lib():
         L.sirllm_step.argtypes = [cfgp] + [vp] * 14
         L.sirllm_step_phases.restype = ctypes.c_int
         L.sirllm_step_phases.argtypes = [cfgp] + [vp] * 14 + [ctypes.POINTER(vp)]
+        L.sirllm_step_host.restype = ctypes.c_int
+        L.sirllm_step_host.argtypes = [cfgp] + [vp] * 23
         L.sirllm_status.restype = ctypes.c_int
         L.sirllm_status.argtypes = [vp, vp, ctypes.POINTER(i32), i32]
         L.sirllm_strerror.restype = ctypes.c_char_p
@@ -223,6 +226,36 @@ def sirllm_step_phases(cfg: Config, logits, token_ids, n_new, scores, serial, li
                                     _dev(n_keep, torch.int32, "n_keep"),
                                     _dev(new_entropy, torch.float32, "new_entropy"),
                                     _dev(ws, torch.uint8, "ws"), _stream(), handles))
+
+
+def _host(t: Optional[torch.Tensor], dtype=None, name="tensor") -> Optional[int]:
+    if t is None:
+        return None
+    if t.is_cuda or not t.is_contiguous():
+        raise SirllmError(ERR_ALIGN, f"{name} must be a contiguous host tensor")
+    if dtype is not None and t.dtype not in (dtype if isinstance(dtype, tuple) else (dtype,)):
+        raise SirllmError(ERR_BAD_CONFIG, f"{name} has dtype {t.dtype}")
+    return t.data_ptr()
+
+
+def sirllm_step_host(cfg: Config, h_logits, h_token_ids, h_n_new, h_new_k, h_new_v, h_live_len,
+                     d_logits, d_token_ids, d_n_new, scores, serial, live_len, decay, k, v,
+                     keep_idx, n_keep, new_entropy, h_keep_idx, h_n_keep, h_new_entropy, ws) -> None:
+    """One round with HOST inputs and outputs (``h_*`` are CPU tensors, ideally pinned);
+    the results are valid after ``torch.cuda.current_stream().synchronize()``."""
+    ldt = {F32: torch.float32, BF16: torch.bfloat16}[cfg.logits_dtype]
+    _check(lib().sirllm_step_host(
+        ctypes.byref(cfg), _host(h_logits, ldt, "h_logits"), _host(h_token_ids, torch.int32, "h_token_ids"),
+        _host(h_n_new, torch.int32, "h_n_new"), _host(h_new_k, _KV, "h_new_k"),
+        _host(h_new_v, _KV, "h_new_v"), _host(h_live_len, torch.int32, "h_live_len"),
+        _logits_ptr(cfg, d_logits), _dev(d_token_ids, torch.int32, "d_token_ids"),
+        _dev(d_n_new, torch.int32, "d_n_new"), _dev(scores, torch.float32, "scores"),
+        _dev(serial, torch.int64, "serial"), _dev(live_len, torch.int32, "live_len"),
+        _dev(decay, torch.float32, "decay"), _dev(k, _KV, "k"), _dev(v, _KV, "v"),
+        _dev(keep_idx, torch.int32, "keep_idx"), _dev(n_keep, torch.int32, "n_keep"),
+        _dev(new_entropy, torch.float32, "new_entropy"), _host(h_keep_idx, torch.int32, "h_keep_idx"),
+        _host(h_n_keep, torch.int32, "h_n_keep"), _host(h_new_entropy, torch.float32, "h_new_entropy"),
+        _dev(ws, torch.uint8, "ws"), _stream()))
 
 
 def sirllm_status(ws: torch.Tensor, clear: bool = False) -> int:

@@ -256,6 +256,73 @@ int sirllm_step_phases(const sirllm_config* cfg, const void* logits, const int32
                      n_keep, new_entropy, ws, cuda_stream, phase_events);
 }
 
+int sirllm_step_host(const sirllm_config* cfg, const void* h_logits, const int32_t* h_token_ids,
+                     const int32_t* h_n_new, const void* h_new_k, const void* h_new_v,
+                     const int32_t* h_live_len, void* d_logits, int32_t* d_token_ids,
+                     int32_t* d_n_new, float* scores, int64_t* serial, int32_t* live_len,
+                     const float* decay, void* k, void* v, int32_t* keep_idx, int32_t* n_keep,
+                     float* new_entropy, int32_t* h_keep_idx, int32_t* h_n_keep,
+                     float* h_new_entropy, void* ws, void* cuda_stream) {
+    int rc = validate_config(cfg);
+    if (rc != SIRLLM_OK) return rc;
+    if (!h_logits || !h_token_ids || !h_n_new || !h_live_len || !d_logits || !d_token_ids ||
+        !d_n_new || !keep_idx || !n_keep || !new_entropy || !h_keep_idx || !h_n_keep ||
+        !h_new_entropy)
+        return SIRLLM_ERR_NULL;
+    if ((h_new_k != nullptr && k == nullptr) || (h_new_v != nullptr && v == nullptr))
+        return SIRLLM_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t es = (size_t)logits_elem_bytes(cfg->logits_dtype);
+    const size_t row_bytes = (size_t)cfg->head_dim * 2;
+    const size_t planes = (size_t)cfg->n_layers * cfg->n_kv_heads;
+    cudaError_t e;
+    for (int s = 0; s < cfg->n_streams; ++s) {
+        const int T = h_n_new[s], l = h_live_len[s];
+        if (T < 0 || T > cfg->max_new || l < 0) return SIRLLM_ERR_BAD_CONFIG;
+        if (T == 0 || l + T > cfg->capacity) continue;  // the device skips and flags an overflow
+        const size_t row0 = (size_t)s * cfg->max_new;
+        if (cfg->logits_row_stride == cfg->vocab) {
+            e = cudaMemcpyAsync((char*)d_logits + row0 * cfg->vocab * es,
+                                (const char*)h_logits + row0 * cfg->vocab * es,
+                                (size_t)T * cfg->vocab * es, cudaMemcpyHostToDevice, st);
+        } else {
+            e = cudaMemcpy2DAsync((char*)d_logits + row0 * cfg->logits_row_stride * es,
+                                  cfg->logits_row_stride * es,
+                                  (const char*)h_logits + row0 * cfg->logits_row_stride * es,
+                                  cfg->logits_row_stride * es, cfg->vocab * es, T,
+                                  cudaMemcpyHostToDevice, st);
+        }
+        if (e != cudaSuccess) return cuda_fail(e, "logits H2D");
+        const void* hsrc[2] = {h_new_k, h_new_v};
+        void* ddst[2] = {k, v};
+        for (int c = 0; c < 2; ++c) {
+            if (!hsrc[c]) continue;
+            e = cudaMemcpy2DAsync((char*)ddst[c] + ((size_t)s * planes * cfg->capacity + l) * row_bytes,
+                                  (size_t)cfg->capacity * row_bytes,
+                                  (const char*)hsrc[c] + (size_t)s * planes * cfg->max_new * row_bytes,
+                                  (size_t)cfg->max_new * row_bytes, (size_t)T * row_bytes, planes,
+                                  cudaMemcpyHostToDevice, st);
+            if (e != cudaSuccess) return cuda_fail(e, "K/V H2D");
+        }
+    }
+    const size_t n_rows = (size_t)cfg->n_streams * cfg->max_new;
+    e = cudaMemcpyAsync(d_token_ids, h_token_ids, n_rows * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e, "ids H2D");
+    e = cudaMemcpyAsync(d_n_new, h_n_new, (size_t)cfg->n_streams * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e, "n_new H2D");
+    rc = step_impl(cfg, d_logits, d_token_ids, d_n_new, scores, serial, live_len, decay, k, v,
+                   keep_idx, n_keep, new_entropy, ws, cuda_stream, nullptr);
+    if (rc != SIRLLM_OK) return rc;
+    e = cudaMemcpyAsync(h_keep_idx, keep_idx, (size_t)cfg->n_streams * cfg->threshold * 4,
+                        cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "keep D2H");
+    e = cudaMemcpyAsync(h_n_keep, n_keep, (size_t)cfg->n_streams * 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "n_keep D2H");
+    e = cudaMemcpyAsync(h_new_entropy, new_entropy, n_rows * 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "entropy D2H");
+    return SIRLLM_OK;
+}
+
 int sirllm_status(void* ws, void* cuda_stream, int32_t* status_out, int32_t clear) {
     if (!ws || !status_out) return SIRLLM_ERR_NULL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
