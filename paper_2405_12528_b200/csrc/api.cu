@@ -49,6 +49,8 @@ WorkspaceLayout workspace_layout(const sirllm_config& c) {
     off = align_up(off + (size_t)c.n_streams * 4, 256);
     L.keep_off = off;
     off = align_up(off + (size_t)c.n_streams * c.threshold * 4, 256);
+    L.tickets_off = off;
+    off = align_up(off + (size_t)c.n_streams * c.max_new * 4, 256);
     L.partials_off = off;
     off = align_up(off + (size_t)c.n_streams * c.max_new * L.n_seg * sizeof(float2), 256);
     L.total = off;
@@ -64,6 +66,12 @@ static ScoreParams score_params(const sirllm_config& c, const WorkspaceLayout& L
     sp.token_ids = ids;
     sp.n_new = n_new;
     sp.partials = (float2*)((char*)ws + L.partials_off);
+    sp.tickets = (int32_t*)((char*)ws + L.tickets_off);
+    sp.status = (int32_t*)ws;
+    sp.out_entropy = nullptr;
+    sp.scores = nullptr;
+    sp.live_len = nullptr;
+    sp.capacity = c.capacity;
     sp.vocab = c.vocab;
     sp.row_stride = c.logits_row_stride;
     sp.n_streams = c.n_streams;
@@ -106,13 +114,10 @@ int sirllm_score(const sirllm_config* cfg, const void* logits, const int32_t* to
     if (misaligned(ws, 256)) return SIRLLM_ERR_ALIGN;
     if ((rc = check_logits(*cfg, logits)) != SIRLLM_OK) return rc;
     const WorkspaceLayout L = workspace_layout(*cfg);
-    const ScoreParams sp = score_params(*cfg, L, logits, token_ids, n_new, ws);
-    cudaStream_t st = (cudaStream_t)cuda_stream;
-    cudaError_t e = launch_score_partials(sp, st);
-    if (e != cudaSuccess) return cuda_fail(e, "score_partials");
-    e = launch_score_finalize(sp, out_entropy, (int32_t*)ws, st);
-    if (e != cudaSuccess) return cuda_fail(e, "score_finalize");
-    return SIRLLM_OK;
+    ScoreParams sp = score_params(*cfg, L, logits, token_ids, n_new, ws);
+    sp.out_entropy = out_entropy;
+    cudaError_t e = launch_score(sp, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "score");
 }
 
 static SelectParams select_params(const sirllm_config& c, const WorkspaceLayout& L, float* scores,
@@ -211,8 +216,12 @@ static int step_impl(const sirllm_config* cfg, const void* logits, const int32_t
     if ((rc = check_logits(*cfg, logits)) != SIRLLM_OK) return rc;
     const WorkspaceLayout L = workspace_layout(*cfg);
     SelectParams sp = select_params(*cfg, L, scores, serial, live_len, decay, keep_idx, n_keep, ws);
-    sp.sc = score_params(*cfg, L, logits, token_ids, n_new, ws);
-    sp.new_entropy = new_entropy;
+    ScoreParams sc = score_params(*cfg, L, logits, token_ids, n_new, ws);
+    sc.out_entropy = new_entropy;
+    sc.scores = scores;
+    sc.live_len = live_len;
+    sp.n_new = n_new;
+    sp.max_new = cfg->max_new;
     sp.compact_scores = 1;
     sp.score_new = 1;
     CompactParams cp;
@@ -224,8 +233,8 @@ static int step_impl(const sirllm_config* cfg, const void* logits, const int32_t
     if (ev && (e = cudaEventRecord((cudaEvent_t)ev[i], st)) != cudaSuccess) \
         return cuda_fail(e, "cudaEventRecord");
     SIRLLM_MARK(0)
-    e = launch_score_partials(sp.sc, st);
-    if (e != cudaSuccess) return cuda_fail(e, "score_partials");
+    e = launch_score(sc, st);
+    if (e != cudaSuccess) return cuda_fail(e, "score");
     SIRLLM_MARK(1)
     e = launch_select(sp, cfg->n_streams, st);
     if (e != cudaSuccess) return cuda_fail(e, "select");

@@ -13,11 +13,13 @@ namespace sirllm {
 //   first_moved[n_streams]                first slot whose row changes place when compacting
 //   n_keep_fallback[n_streams]            used when the caller passes no n_keep
 //   keep_fallback[n_streams][threshold]   used when the caller passes no keep_idx
+//   tickets[n_streams*max_new]            arrivals per logits row (the last segment finishes the row)
 //   partials[n_streams*max_new][n_seg]    (scaled max, sum) pairs of the split log-sum-exp
 struct WorkspaceLayout {
     size_t first_moved_off;
     size_t n_keep_off;
     size_t keep_off;
+    size_t tickets_off;
     size_t partials_off;
     size_t total;
     int32_t n_seg;  // vocabulary segments per logits row
@@ -40,14 +42,19 @@ struct ScoreParams {
     const int32_t* token_ids;
     const int32_t* n_new;  // nullable: max_new for every stream
     float2* partials;
+    int32_t* tickets;
+    int32_t* status;
+    float* out_entropy;        // [n_streams*max_new] raw scores, nullable
+    float* scores;             // nullable: also append at scores[s][live_len[s] + t] (fused round)
+    const int32_t* live_len;   // with `scores`
     int64_t vocab;
     int64_t row_stride;
-    int32_t n_streams, max_new, n_seg, logits_dtype;
+    int32_t n_streams, max_new, n_seg, logits_dtype, capacity;
 };
 
 struct SelectParams {
-    ScoreParams sc;        // used when score_new != 0
-    float* new_entropy;    // nullable
+    const int32_t* n_new;  // with score_new: tokens appended this round (nullable: max_new)
+    int32_t max_new;
     float* scores;
     int64_t* serial;       // nullable
     int32_t* live_len;
@@ -58,7 +65,7 @@ struct SelectParams {
     int32_t* status;
     int32_t capacity, budget, n_sink, n_recent, threshold;
     int32_t compact_scores;  // also gather scores / serial and commit live_len
-    int32_t score_new;       // finish and append the scores of the round's new tokens first
+    int32_t score_new;       // the round's new scores were appended behind live_len by the scorer
 };
 
 struct CompactParams {
@@ -74,9 +81,7 @@ struct CompactParams {
     int32_t in_place;
 };
 
-cudaError_t launch_score_partials(const ScoreParams& p, cudaStream_t st);
-cudaError_t launch_score_finalize(const ScoreParams& p, float* out_entropy, int32_t* status,
-                                  cudaStream_t st);
+cudaError_t launch_score(const ScoreParams& p, cudaStream_t st);
 cudaError_t launch_select(const SelectParams& p, int n_streams, cudaStream_t st);
 cudaError_t launch_compact_plan(const CompactParams& p, int n_streams, int32_t* first_moved,
                                 cudaStream_t st);
@@ -98,18 +103,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // larger score; negatives sort below non-negatives and -0 below +0.
 __device__ __forceinline__ uint32_t order_key(uint32_t bits) {
     return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
-}
-
-// Combine the per-segment (scaled max M, sum S) pairs of one logits row, where
-// sum_v exp(z_v) = S * 2^M, and return the token's entropy  ln(sum exp z) - z_id  (>= 0).
-__device__ __forceinline__ float finish_entropy(const float2* __restrict__ part, int n_seg,
-                                                float z_id) {
-    float M = kNegHuge;
-    for (int i = 0; i < n_seg; ++i) M = fmaxf(M, part[i].x);
-    double S = 0.0;
-    for (int i = 0; i < n_seg; ++i) S += (double)part[i].y * exp2((double)part[i].x - (double)M);
-    double e = ((double)M * kLn2 + log(S)) - (double)z_id;
-    return fmaxf((float)e, 0.0f);
 }
 
 __device__ __forceinline__ float load_logit(const void* logits, int dtype, int64_t idx) {

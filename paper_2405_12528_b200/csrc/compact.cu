@@ -139,14 +139,17 @@ compact_kernel(const CompactParams p, const int stages, const int n_units) {
         int f = p.first_moved[s];
         if (f < 0) continue;  // keep list rejected
         if (!p.in_place) f = 0;
-        const char* src = p.src[tensor] + (size_t)plane * p.capacity * p.row_bytes;
-        char* dst = p.dst[tensor] + (size_t)plane * p.capacity * p.row_bytes;
+        const char* src = (tensor ? p.src[1] : p.src[0]) + (size_t)plane * p.capacity * p.row_bytes;
+        char* dst = (tensor ? p.dst[1] : p.dst[0]) + (size_t)plane * p.capacity * p.row_bytes;
         const int32_t* keep = p.keep_idx + (size_t)s * p.keep_stride;
 
+        int kj_next = f + lane < n ? keep[f + lane] : -2;  // source rows of the first chunk
         for (int j0 = f; j0 < n && alive; j0 += kChunkRows) {
             const int nrows = min(kChunkRows, n - j0);
             const int stage = (int)(it % stages);
-            const int kj = lane < nrows ? keep[j0 + lane] : -2;
+            const int kj = kj_next;
+            // fetch the next chunk's source rows now; they are needed one trip later
+            kj_next = j0 + kChunkRows + lane < n ? keep[j0 + kChunkRows + lane] : -2;
             if (lane == 0) {
                 if (it >= stages) bulk_wait_read<kStoreSlack>();  // the stage's last store has left
                 ring.st_dst[stage] = dst + (size_t)j0 * p.row_bytes;

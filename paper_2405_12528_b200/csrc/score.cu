@@ -1,8 +1,9 @@
 // Token Entropy (Section 3.2): e = -log softmax(z)[id] as a vocabulary-streaming
 // log-sum-exp.  Every logits row is cut into segments of kVecPerSeg 16-byte vectors;
 // one warp reduces one segment with an online (running-max) softmax sum and writes a
-// (scaled max, sum) pair.  The pairs of a row are combined in fp64 by whoever needs the
-// score: score_finalize_kernel here, or the selection kernel in the fused round.
+// (scaled max, sum) pair to scratch.  The warp that arrives last on the row's ticket
+// combines the row's pairs in fp64 (in a fixed order, so the result does not depend on
+// which warp that is), writes the score and, in the fused round, appends it to E.
 //
 // The kernel is bound by HBM reads (2 or 4 bytes per element, each read once); the
 // arithmetic per element is one conversion, one max, one FMA, one ex2 and one add.
@@ -52,7 +53,7 @@ __device__ __forceinline__ uint32_t bf162_max(uint32_t a, uint32_t b) {
 
 template <bool kBf16>
 __global__ void __launch_bounds__(kScoreWarpsPerCta * 32)
-score_partials_kernel(const ScoreParams p) {
+score_kernel(const ScoreParams p) {
     constexpr int ES = kBf16 ? 2 : 4;
     constexpr int EPV = 16 / ES;
     const int lane = threadIdx.x & 31;
@@ -63,9 +64,26 @@ score_partials_kernel(const ScoreParams p) {
     const int64_t row = warp / p.n_seg;
     const int s = (int)(row / p.max_new);
     const int t = (int)(row - (int64_t)s * p.max_new);
-    if (p.n_new != nullptr && t >= p.n_new[s]) return;
-
+    int T = p.max_new;
+    if (p.n_new != nullptr) T = min(p.n_new[s], p.max_new);
+    if (t >= T) return;
     const int64_t V = p.vocab;
+    const int32_t id = p.token_ids[row];
+    // where the fused round appends this token's score (nowhere if the round does not fit)
+    float* append = nullptr;
+    if (p.scores != nullptr) {
+        const int l0 = p.live_len[s];
+        if (l0 >= 0 && l0 <= p.capacity - T) append = p.scores + (size_t)s * p.capacity + l0 + t;
+    }
+    if (id < 0 || (int64_t)id >= V) {  // no prediction for this position, or a bad id: score 0
+        if (seg == 0 && lane == 0) {
+            if (id != -1) atomicOr(p.status, SIRLLM_STATUS_TOKEN_RANGE);
+            if (p.out_entropy) p.out_entropy[row] = 0.f;
+            if (append) *append = 0.f;
+        }
+        return;
+    }
+
     const char* rowp = (const char*)p.logits + row * p.row_stride * ES;
     // elements in front of the first 16-byte boundary, whole vectors, elements after them
     int64_t head = (int64_t)(((16u - (uint32_t)((uintptr_t)rowp & 15u)) & 15u) / ES);
@@ -138,45 +156,48 @@ score_partials_kernel(const ScoreParams p) {
     float S = (st.s0 + st.s1) * ex2_approx(st.mL - M);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(0xFFFFFFFFu, S, o);
-    if (lane == 0) p.partials[row * p.n_seg + seg] = make_float2(M, S);
-}
-
-__global__ void score_finalize_kernel(const ScoreParams p, float* __restrict__ out,
-                                      int32_t* __restrict__ status) {
-    const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (row >= (int64_t)p.n_streams * p.max_new) return;
-    const int s = (int)(row / p.max_new);
-    const int t = (int)(row - (int64_t)s * p.max_new);
-    if (p.n_new != nullptr && t >= p.n_new[s]) return;
-    const int32_t id = p.token_ids[row];
-    float e = 0.f;
-    if (id >= 0 && (int64_t)id < p.vocab) {
-        const float z = load_logit(p.logits, p.logits_dtype, row * p.row_stride + id);
-        e = finish_entropy(p.partials + row * p.n_seg, p.n_seg, z);
-    } else if (id != -1) {
-        atomicOr(status, SIRLLM_STATUS_TOKEN_RANGE);
+    // publish the pair; the last of the row's warps to arrive finishes the row
+    float2* part = p.partials + row * p.n_seg;
+    int arrived = 0;
+    if (lane == 0) {
+        part[seg] = make_float2(M, S);
+        __threadfence();
+        arrived = atomicAdd(&p.tickets[row], 1);
     }
-    out[row] = e;
+    arrived = __shfl_sync(0xFFFFFFFFu, arrived, 0);
+    if (arrived != p.n_seg - 1) return;
+    __threadfence();
+    if (lane == 0) p.tickets[row] = 0;  // ready for the next call
+    float Mx = kNegHuge;
+    for (int i = lane; i < p.n_seg; i += 32) Mx = fmaxf(Mx, __ldcg(&part[i]).x);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) Mx = fmaxf(Mx, __shfl_xor_sync(0xFFFFFFFFu, Mx, o));
+    double acc = 0.0;
+    for (int i = lane; i < p.n_seg; i += 32) {
+        const float2 q = __ldcg(&part[i]);
+        acc += (double)q.y * exp2((double)q.x - (double)Mx);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    if (lane == 0) {
+        // sum_v exp(z_v) = acc * 2^Mx;  e = ln(sum) - z_id >= 0
+        const float z = load_logit(rowp, kBf16 ? SIRLLM_BF16 : SIRLLM_F32, id);
+        const float e = fmaxf((float)(((double)Mx * kLn2 + log(acc)) - (double)z), 0.0f);
+        if (p.out_entropy) p.out_entropy[row] = e;
+        if (append) *append = e;
+    }
 }
 
 }  // namespace
 
-cudaError_t launch_score_partials(const ScoreParams& p, cudaStream_t st) {
+cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
     const int64_t warps = (int64_t)p.n_streams * p.max_new * p.n_seg;
     if (warps == 0) return cudaSuccess;
     const unsigned grid = (unsigned)((warps + kScoreWarpsPerCta - 1) / kScoreWarpsPerCta);
     if (p.logits_dtype == SIRLLM_BF16)
-        score_partials_kernel<true><<<grid, kScoreWarpsPerCta * 32, 0, st>>>(p);
+        score_kernel<true><<<grid, kScoreWarpsPerCta * 32, 0, st>>>(p);
     else
-        score_partials_kernel<false><<<grid, kScoreWarpsPerCta * 32, 0, st>>>(p);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_score_finalize(const ScoreParams& p, float* out_entropy, int32_t* status,
-                                  cudaStream_t st) {
-    const int64_t rows = (int64_t)p.n_streams * p.max_new;
-    if (rows == 0) return cudaSuccess;
-    score_finalize_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, st>>>(p, out_entropy, status);
+        score_kernel<false><<<grid, kScoreWarpsPerCta * 32, 0, st>>>(p);
     return cudaGetLastError();
 }
 

@@ -63,9 +63,9 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
 
     const int l0 = p.live_len[s];
     int T = 0;
-    if (p.score_new) {
-        T = p.sc.n_new ? p.sc.n_new[s] : p.sc.max_new;
-        T = max(0, min(T, p.sc.max_new));
+    if (p.score_new) {  // the scorer has appended T raw scores behind slot l0
+        T = p.n_new ? p.n_new[s] : p.max_new;
+        T = max(0, min(T, p.max_new));
     }
     if (l0 < 0 || l0 > cap - T) {  // the round does not fit: leave the stream alone
         if (tid == 0) {
@@ -78,29 +78,12 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     }
     const int l = l0 + T;
 
-    // ---- S1 (tail) + S2: finish the new tokens' scores and append them --------------
-    for (int t = tid; t < T; t += kSelectThreads) {
-        const int64_t row = (int64_t)s * p.sc.max_new + t;
-        const int32_t id = p.sc.token_ids[row];
-        float e = 0.f;
-        if (id >= 0 && (int64_t)id < p.sc.vocab) {
-            const float z = load_logit(p.sc.logits, p.sc.logits_dtype, row * p.sc.row_stride + id);
-            e = finish_entropy(p.sc.partials + row * p.sc.n_seg, p.sc.n_seg, z);
-        } else if (id != -1) {
-            atomicOr(p.status, SIRLLM_STATUS_TOKEN_RANGE);
-        }
-        if (p.new_entropy) p.new_entropy[row] = e;
-        vals[l0 + t] = __float_as_uint(e);
-    }
-    __syncthreads();
-
     // ---- S3: one fp32 multiply per held score -----------------------------------------
     const float eta = p.decay[s];
     const bool evict = l > p.threshold;
     const bool write_now = !(evict && p.compact_scores);
     for (int i = tid; i < l; i += kSelectThreads) {
-        float x = i < l0 ? scores[i] : __uint_as_float(vals[i]);
-        x = __fmul_rn(x, eta);
+        const float x = __fmul_rn(scores[i], eta);
         vals[i] = __float_as_uint(x);
         if (write_now) scores[i] = x;
     }

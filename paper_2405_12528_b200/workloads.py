@@ -148,6 +148,10 @@ WORKLOADS = {
                           "bf16", "bf16", 0.9, 20, zipf_bias=1.1),
     "batched64": Workload("batched64", 64, 32, 32, 128, 2048, 1024, 4, 256, 256, 32000,
                           "bf16", "bf16", 0.7, 100, decay_hi=1.0),
+    # A quarter of llama3_8b in tokens and slots (same vocabulary, planes and row size): the
+    # small case profiler captures run on.
+    "llama3_8b_quarter": Workload("llama3_8b_quarter", 1, 32, 8, 128, 4096, 2048, 4, 256, 1024,
+                                  128256, "bf16", "bf16", 0.9, 20, zipf_bias=1.1),
     # Shapes the paper's own runs had (Tables 1-3, 5-7): small rounds, no recent window.
     "rps_1024": Workload("rps_1024", 1, 32, 32, 128, 1152, 1024, 4, 0, 54, 32000,
                          "bf16", "bf16", 0.8, 2000),
