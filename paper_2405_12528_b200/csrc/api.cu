@@ -40,8 +40,9 @@ WorkspaceLayout workspace_layout(const sirllm_config& c) {
     WorkspaceLayout L;
     const int64_t epv = 16 / logits_elem_bytes(c.logits_dtype);
     const int64_t nvec = c.vocab / epv;
-    L.n_seg = (int32_t)((nvec + kVecPerSeg - 1) / kVecPerSeg);
-    if (L.n_seg < 1) L.n_seg = 1;
+    const int64_t per_cta = (int64_t)kVecPerSeg * kScoreWarpsPerCta;
+    L.n_part = (int32_t)((nvec + per_cta - 1) / per_cta);
+    if (L.n_part < 1) L.n_part = 1;
     size_t off = 256;
     L.first_moved_off = off;
     off = align_up(off + (size_t)c.n_streams * 4, 256);
@@ -52,7 +53,7 @@ WorkspaceLayout workspace_layout(const sirllm_config& c) {
     L.tickets_off = off;
     off = align_up(off + (size_t)c.n_streams * c.max_new * 4, 256);
     L.partials_off = off;
-    off = align_up(off + (size_t)c.n_streams * c.max_new * L.n_seg * sizeof(float2), 256);
+    off = align_up(off + (size_t)c.n_streams * c.max_new * L.n_part * sizeof(float2), 256);
     L.total = off;
     return L;
 }
@@ -76,7 +77,7 @@ static ScoreParams score_params(const sirllm_config& c, const WorkspaceLayout& L
     sp.row_stride = c.logits_row_stride;
     sp.n_streams = c.n_streams;
     sp.max_new = c.max_new;
-    sp.n_seg = L.n_seg;
+    sp.n_part = L.n_part;
     sp.logits_dtype = c.logits_dtype;
     return sp;
 }
@@ -152,7 +153,7 @@ int sirllm_decay_select(const sirllm_config* cfg, float* scores, int64_t* serial
     SelectParams p = select_params(*cfg, L, scores, serial, live_len, decay, keep_idx, n_keep, ws);
     p.compact_scores = compact_scores != 0;
     p.score_new = 0;
-    cudaError_t e = launch_select(p, cfg->n_streams, (cudaStream_t)cuda_stream);
+    cudaError_t e = launch_select(p, cfg->n_streams, (cudaStream_t)cuda_stream, false);
     return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "select");
 }
 
@@ -201,7 +202,7 @@ int sirllm_compact_kv(const sirllm_config* cfg, const void* k_src, const void* v
     cudaStream_t st = (cudaStream_t)cuda_stream;
     cudaError_t e = launch_compact_plan(p, cfg->n_streams, (int32_t*)((char*)ws + L.first_moved_off), st);
     if (e != cudaSuccess) return cuda_fail(e, "compact_plan");
-    e = launch_compact(p, st);
+    e = launch_compact(p, st, true);
     return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "compact");
 }
 
@@ -236,10 +237,10 @@ static int step_impl(const sirllm_config* cfg, const void* logits, const int32_t
     e = launch_score(sc, st);
     if (e != cudaSuccess) return cuda_fail(e, "score");
     SIRLLM_MARK(1)
-    e = launch_select(sp, cfg->n_streams, st);
+    e = launch_select(sp, cfg->n_streams, st, ev == nullptr);
     if (e != cudaSuccess) return cuda_fail(e, "select");
     SIRLLM_MARK(2)
-    e = launch_compact(cp, st);
+    e = launch_compact(cp, st, ev == nullptr);
     if (e != cudaSuccess) return cuda_fail(e, "compact");
     SIRLLM_MARK(3)
 #undef SIRLLM_MARK

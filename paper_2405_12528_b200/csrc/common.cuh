@@ -13,8 +13,8 @@ namespace sirllm {
 //   first_moved[n_streams]                first slot whose row changes place when compacting
 //   n_keep_fallback[n_streams]            used when the caller passes no n_keep
 //   keep_fallback[n_streams][threshold]   used when the caller passes no keep_idx
-//   tickets[n_streams*max_new]            arrivals per logits row (the last segment finishes the row)
-//   partials[n_streams*max_new][n_seg]    (scaled max, sum) pairs of the split log-sum-exp
+//   tickets[n_streams*max_new]            arrivals per logits row (the last CTA finishes the row)
+//   partials[n_streams*max_new][n_part]   (scaled max, sum) pair per CTA of a multi-CTA row
 struct WorkspaceLayout {
     size_t first_moved_off;
     size_t n_keep_off;
@@ -22,7 +22,7 @@ struct WorkspaceLayout {
     size_t tickets_off;
     size_t partials_off;
     size_t total;
-    int32_t n_seg;  // vocabulary segments per logits row
+    int32_t n_part;  // CTAs (groups of kScoreWarpsPerCta segments) per logits row
 };
 
 constexpr int kVecPerSeg = 512;  // 16-byte vectors per segment: 8 KB of logits per warp
@@ -49,7 +49,7 @@ struct ScoreParams {
     const int32_t* live_len;   // with `scores`
     int64_t vocab;
     int64_t row_stride;
-    int32_t n_streams, max_new, n_seg, logits_dtype, capacity;
+    int32_t n_streams, max_new, n_part, logits_dtype, capacity;
 };
 
 struct SelectParams {
@@ -82,16 +82,29 @@ struct CompactParams {
 };
 
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st);
-cudaError_t launch_select(const SelectParams& p, int n_streams, cudaStream_t st);
+// `overlap`: launch with programmatic stream serialization, so the grid may become resident
+// while the previous kernel on the stream drains; the kernel itself waits for that kernel's
+// results (grid_dependency_wait) before it reads them.
+cudaError_t launch_select(const SelectParams& p, int n_streams, cudaStream_t st, bool overlap);
 cudaError_t launch_compact_plan(const CompactParams& p, int n_streams, int32_t* first_moved,
                                 cudaStream_t st);
-cudaError_t launch_compact(const CompactParams& p, cudaStream_t st);
+cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap);
 
 // ---- small device helpers ----------------------------------------------------------------
 #ifdef __CUDACC__
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr double kLn2 = 0.6931471805599453;
 constexpr float kNegHuge = -3.0e38f;  // "no element seen yet" for a running maximum
+
+// Programmatic dependent launch: wait until the preceding kernel on the stream has
+// completed and its writes are visible (no-op for a normally launched kernel); allow the
+// following kernel to start becoming resident.
+__device__ __forceinline__ void grid_dependency_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void grid_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;

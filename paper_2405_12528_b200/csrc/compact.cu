@@ -123,6 +123,7 @@ compact_kernel(const CompactParams p, const int stages, const int n_units) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncwarp();
+    grid_dependency_wait();  // the keep lists of the selection kernel
 
     const int lead = stages - 1 - kStoreSlack;  // chunks whose loads run ahead of the stores
     const int64_t g = (int64_t)blockIdx.x * n_workers + wid;
@@ -221,7 +222,7 @@ cudaError_t launch_compact_plan(const CompactParams& p, int n_streams, int32_t* 
     return cudaGetLastError();
 }
 
-cudaError_t launch_compact(const CompactParams& p, cudaStream_t st) {
+cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap) {
     int n_tensors = 0;
     CompactParams q = p;
     for (int t = 0; t < 2; ++t) {
@@ -259,8 +260,17 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     const int grid = (int)((n_units + workers - 1) / workers < n_sm ? (n_units + workers - 1) / workers
                                                                     : n_sm);
-    compact_kernel<<<grid, workers * 32, smem, st>>>(q, stages, n_units);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)workers * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, compact_kernel, q, stages, n_units);
 }
 
 }  // namespace sirllm

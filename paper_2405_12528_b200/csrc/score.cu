@@ -1,9 +1,12 @@
 // Token Entropy (Section 3.2): e = -log softmax(z)[id] as a vocabulary-streaming
 // log-sum-exp.  Every logits row is cut into segments of kVecPerSeg 16-byte vectors;
-// one warp reduces one segment with an online (running-max) softmax sum and writes a
-// (scaled max, sum) pair to scratch.  The warp that arrives last on the row's ticket
-// combines the row's pairs in fp64 (in a fixed order, so the result does not depend on
-// which warp that is), writes the score and, in the fused round, appends it to E.
+// one warp reduces one segment with an online (running-max) softmax sum, and the
+// kScoreWarpsPerCta warps of a CTA (consecutive segments of one row) combine their
+// (scaled max, sum) pairs through shared memory.  A row that needs several CTAs
+// (vocabularies above 32768 bf16 / 16384 fp32 elements) publishes one pair per CTA in
+// scratch; the CTA that arrives last on the row's ticket combines them.  Combination is
+// in fp64 and in a fixed order, so the score does not depend on which CTA comes last.
+// The finishing warp writes the score and, in the fused round, appends it to E.
 //
 // The kernel is bound by HBM reads (2 or 4 bytes per element, each read once); the
 // arithmetic per element is one conversion, one max, one FMA, one ex2 and one add.
@@ -56,34 +59,27 @@ __global__ void __launch_bounds__(kScoreWarpsPerCta * 32)
 score_kernel(const ScoreParams p) {
     constexpr int ES = kBf16 ? 2 : 4;
     constexpr int EPV = 16 / ES;
-    const int lane = threadIdx.x & 31;
-    const int64_t warp = (int64_t)blockIdx.x * kScoreWarpsPerCta + (threadIdx.x >> 5);
-    const int64_t total = (int64_t)p.n_streams * p.max_new * p.n_seg;
-    if (warp >= total) return;
-    const int seg = (int)(warp % p.n_seg);
-    const int64_t row = warp / p.n_seg;
+    __shared__ float2 warp_pair[kScoreWarpsPerCta];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    grid_launch_dependents();
+    // one CTA = kScoreWarpsPerCta consecutive segments of one logits row
+    const int64_t row = blockIdx.x / p.n_part;
+    const int part_idx = (int)(blockIdx.x - row * p.n_part);
+    const int seg = part_idx * kScoreWarpsPerCta + wid;
     const int s = (int)(row / p.max_new);
     const int t = (int)(row - (int64_t)s * p.max_new);
     int T = p.max_new;
     if (p.n_new != nullptr) T = min(p.n_new[s], p.max_new);
     if (t >= T) return;
-    const int64_t V = p.vocab;
-    const int32_t id = p.token_ids[row];
-    // where the fused round appends this token's score (nowhere if the round does not fit)
-    float* append = nullptr;
-    if (p.scores != nullptr) {
-        const int l0 = p.live_len[s];
-        if (l0 >= 0 && l0 <= p.capacity - T) append = p.scores + (size_t)s * p.capacity + l0 + t;
-    }
-    if (id < 0 || (int64_t)id >= V) {  // no prediction for this position, or a bad id: score 0
-        if (seg == 0 && lane == 0) {
-            if (id != -1) atomicOr(p.status, SIRLLM_STATUS_TOKEN_RANGE);
-            if (p.out_entropy) p.out_entropy[row] = 0.f;
-            if (append) *append = 0.f;
-        }
-        return;
+    // warp 0 finishes the row: fetch what it will need now, use it after the reduction
+    int32_t id = -1;
+    int l0 = -1;
+    if (wid == 0) {
+        id = p.token_ids[row];
+        if (p.scores != nullptr) l0 = p.live_len[s];
     }
 
+    const int64_t V = p.vocab;
     const char* rowp = (const char*)p.logits + row * p.row_stride * ES;
     // elements in front of the first 16-byte boundary, whole vectors, elements after them
     int64_t head = (int64_t)(((16u - (uint32_t)((uintptr_t)rowp & 15u)) & 15u) / ES);
@@ -149,51 +145,74 @@ score_kernel(const ScoreParams p) {
         st.raise(z);
         st.add0(z);
     }
-    // warp combine
+    // warp combine -> one (scaled max, sum) pair per warp
     float M = st.mL;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, o));
     float S = (st.s0 + st.s1) * ex2_approx(st.mL - M);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(0xFFFFFFFFu, S, o);
-    // publish the pair; the last of the row's warps to arrive finishes the row
-    float2* part = p.partials + row * p.n_seg;
-    int arrived = 0;
-    if (lane == 0) {
-        part[seg] = make_float2(M, S);
-        __threadfence();
-        arrived = atomicAdd(&p.tickets[row], 1);
-    }
-    arrived = __shfl_sync(0xFFFFFFFFu, arrived, 0);
-    if (arrived != p.n_seg - 1) return;
-    __threadfence();
-    if (lane == 0) p.tickets[row] = 0;  // ready for the next call
-    float Mx = kNegHuge;
-    for (int i = lane; i < p.n_seg; i += 32) Mx = fmaxf(Mx, __ldcg(&part[i]).x);
+    if (lane == 0) warp_pair[wid] = make_float2(M, S);
+    __syncthreads();
+    if (wid != 0) return;
+
+    // CTA combine in fp64 (fixed order): sum_v exp(z_v) over the CTA's segments = acc * 2^Mx
+    float2 q = lane < kScoreWarpsPerCta ? warp_pair[lane] : make_float2(kNegHuge, 0.f);
+    float Mx = q.x;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) Mx = fmaxf(Mx, __shfl_xor_sync(0xFFFFFFFFu, Mx, o));
-    double acc = 0.0;
-    for (int i = lane; i < p.n_seg; i += 32) {
-        const float2 q = __ldcg(&part[i]);
-        acc += (double)q.y * exp2((double)q.x - (double)Mx);
-    }
+    double acc = (double)q.y * exp2((double)q.x - (double)Mx);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+
+    if (p.n_part > 1) {
+        // publish; the CTA that arrives last on the row's ticket combines the row
+        float2* part = p.partials + row * p.n_part;
+        int arrived = 0;
+        if (lane == 0) {
+            part[part_idx] = make_float2(Mx, (float)acc);
+            __threadfence();
+            arrived = atomicAdd(&p.tickets[row], 1);
+        }
+        arrived = __shfl_sync(0xFFFFFFFFu, arrived, 0);
+        if (arrived != p.n_part - 1) return;
+        __threadfence();
+        if (lane == 0) p.tickets[row] = 0;  // ready for the next call
+        Mx = kNegHuge;
+        for (int i = lane; i < p.n_part; i += 32) Mx = fmaxf(Mx, __ldcg(&part[i]).x);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) Mx = fmaxf(Mx, __shfl_xor_sync(0xFFFFFFFFu, Mx, o));
+        acc = 0.0;
+        for (int i = lane; i < p.n_part; i += 32) {
+            const float2 g = __ldcg(&part[i]);
+            acc += (double)g.y * exp2((double)g.x - (double)Mx);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    }
     if (lane == 0) {
-        // sum_v exp(z_v) = acc * 2^Mx;  e = ln(sum) - z_id >= 0
-        const float z = load_logit(rowp, kBf16 ? SIRLLM_BF16 : SIRLLM_F32, id);
-        const float e = fmaxf((float)(((double)Mx * kLn2 + log(acc)) - (double)z), 0.0f);
+        // e = ln(sum_v exp z_v) - z_id >= 0; id -1 = no prediction, other bad ids are flagged
+        float e = 0.f;
+        if (id >= 0 && (int64_t)id < V) {
+            const float z = load_logit(rowp, kBf16 ? SIRLLM_BF16 : SIRLLM_F32, id);
+            e = fmaxf((float)(((double)Mx * kLn2 + log(acc)) - (double)z), 0.0f);
+        } else if (id != -1) {
+            atomicOr(p.status, SIRLLM_STATUS_TOKEN_RANGE);
+        }
         if (p.out_entropy) p.out_entropy[row] = e;
-        if (append) *append = e;
+        // the fused round appends the score behind the live slots (nowhere if it does not fit)
+        if (p.scores != nullptr && l0 >= 0 && l0 <= p.capacity - T)
+            p.scores[(size_t)s * p.capacity + l0 + t] = e;
     }
 }
 
 }  // namespace
 
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
-    const int64_t warps = (int64_t)p.n_streams * p.max_new * p.n_seg;
-    if (warps == 0) return cudaSuccess;
-    const unsigned grid = (unsigned)((warps + kScoreWarpsPerCta - 1) / kScoreWarpsPerCta);
+    const int64_t ctas = (int64_t)p.n_streams * p.max_new * p.n_part;
+    if (ctas == 0) return cudaSuccess;
+    if (ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;
+    const unsigned grid = (unsigned)ctas;
     if (p.logits_dtype == SIRLLM_BF16)
         score_kernel<true><<<grid, kScoreWarpsPerCta * 32, 0, st>>>(p);
     else

@@ -60,6 +60,8 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     const int cap = p.capacity;
     float* scores = p.scores + (size_t)s * cap;
     int32_t* keep = p.keep_idx + (size_t)s * p.threshold;
+    grid_launch_dependents();
+    grid_dependency_wait();  // the scorer's appended scores
 
     const int l0 = p.live_len[s];
     int T = 0;
@@ -227,15 +229,25 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     __syncthreads();
     const int first = sh.first_evicted;
 
-    // ---- S5: the 8-byte tags follow, in place, front to back -------------------------------
+    // ---- S5: the 8-byte tags follow, in place, front to back.  A batch of kTagBatch tags
+    // per thread is read into registers before any of them is written; a later batch only
+    // reads slots at or behind its own first destination, which earlier batches never wrote.
     if (p.serial != nullptr && p.compact_scores) {
+        constexpr int kTagBatch = 8;
         int64_t* serial = p.serial + (size_t)s * cap;
-        for (int base = first; base < p.budget; base += kSelectThreads) {
-            const int j = base + tid;
-            int64_t v = 0;
-            if (j < p.budget) v = serial[keep[j]];
+        for (int base = first; base < p.budget; base += kTagBatch * kSelectThreads) {
+            int64_t v[kTagBatch];
+#pragma unroll
+            for (int q = 0; q < kTagBatch; ++q) {
+                const int j = base + q * kSelectThreads + tid;
+                v[q] = j < p.budget ? serial[keep[j]] : 0;
+            }
             __syncthreads();
-            if (j < p.budget) serial[j] = v;
+#pragma unroll
+            for (int q = 0; q < kTagBatch; ++q) {
+                const int j = base + q * kSelectThreads + tid;
+                if (j < p.budget) serial[j] = v[q];
+            }
             __syncthreads();
         }
     }
@@ -248,17 +260,22 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
 
 }  // namespace
 
-cudaError_t launch_select(const SelectParams& p, int n_streams, cudaStream_t st) {
+cudaError_t launch_select(const SelectParams& p, int n_streams, cudaStream_t st, bool overlap) {
     const size_t smem = (size_t)p.capacity * 4 + (size_t)kRadixBins * 4;
-    static thread_local size_t configured = 0;
-    if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(select_kernel,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = smem;
-    }
-    select_kernel<<<n_streams, kSelectThreads, smem, st>>>(p);
-    return cudaGetLastError();
+    cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)n_streams);
+    cfg.blockDim = dim3(kSelectThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, select_kernel, p);
 }
 
 }  // namespace sirllm
