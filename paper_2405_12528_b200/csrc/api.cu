@@ -44,6 +44,8 @@ WorkspaceLayout workspace_layout(const sirllm_config& c) {
     L.n_part = (int32_t)((nvec + per_cta - 1) / per_cta);
     if (L.n_part < 1) L.n_part = 1;
     size_t off = 256;
+    L.plane_flags_off = off;
+    off = align_up(off + (size_t)2 * c.n_streams * c.n_layers * c.n_kv_heads * 4, 256);
     L.first_moved_off = off;
     off = align_up(off + (size_t)c.n_streams * 4, 256);
     L.n_keep_off = off;
@@ -134,6 +136,7 @@ static SelectParams select_params(const sirllm_config& c, const WorkspaceLayout&
     p.n_keep = n_keep ? n_keep : (int32_t*)((char*)ws + L.n_keep_off);
     p.first_moved = (int32_t*)((char*)ws + L.first_moved_off);
     p.status = (int32_t*)ws;
+    p.epoch = (int32_t*)ws + 1;
     p.capacity = c.capacity;
     p.budget = c.budget;
     p.n_sink = c.n_sink;
@@ -175,6 +178,8 @@ static int compact_params(const sirllm_config& c, const WorkspaceLayout& L, cons
     p.n_keep = n_keep;
     p.first_moved = (int32_t*)((char*)ws + L.first_moved_off);
     p.status = (int32_t*)ws;
+    p.epoch = (int32_t*)ws + 1;
+    p.plane_flags = (int32_t*)((char*)ws + L.plane_flags_off);
     p.planes_per_stream = c.n_layers * c.n_kv_heads;
     p.planes_per_tensor = (int64_t)c.n_streams * p.planes_per_stream;
     p.capacity = c.capacity;

@@ -9,13 +9,15 @@
 namespace sirllm {
 
 // ---- workspace layout (device memory owned by the caller) -------------------------------
-//   [0, 256)                              header: int32 status word
+//   [0, 256)                              header: int32 status word, int32 compaction epoch
+//   plane_flags[2*n_streams*planes]       progress of a plane split across several workers
 //   first_moved[n_streams]                first slot whose row changes place when compacting
 //   n_keep_fallback[n_streams]            used when the caller passes no n_keep
 //   keep_fallback[n_streams][threshold]   used when the caller passes no keep_idx
 //   tickets[n_streams*max_new]            arrivals per logits row (the last CTA finishes the row)
 //   partials[n_streams*max_new][n_part]   (scaled max, sum) pair per CTA of a multi-CTA row
 struct WorkspaceLayout {
+    size_t plane_flags_off;
     size_t first_moved_off;
     size_t n_keep_off;
     size_t keep_off;
@@ -63,6 +65,7 @@ struct SelectParams {
     int32_t* n_keep;
     int32_t* first_moved;
     int32_t* status;
+    int32_t* epoch;
     int32_t capacity, budget, n_sink, n_recent, threshold;
     int32_t compact_scores;  // also gather scores / serial and commit live_len
     int32_t score_new;       // the round's new scores were appended behind live_len by the scorer
@@ -75,6 +78,8 @@ struct CompactParams {
     const int32_t* n_keep;
     const int32_t* first_moved;
     int32_t* status;
+    int32_t* epoch;        // bumped once per compaction by the kernel that precedes it
+    int32_t* plane_flags;  // [tensors * planes_per_tensor]
     int64_t planes_per_tensor;  // n_streams * n_layers * n_kv_heads
     int32_t planes_per_stream;
     int32_t capacity, keep_stride, row_bytes;
@@ -111,6 +116,67 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+
+// ---- mbarrier / TMA bulk-copy wrappers (non-tensor cp.async.bulk: 16-byte aligned
+// addresses, sizes that are multiples of 16 bytes) ------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_init_fence() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t limit) {
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if (++spins > limit) return false;
+    }
+    return true;
+}
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes,
+                                          uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
+            "r"(smem_u32(smem_dst)),
+        "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst),
+                 "r"(smem_u32(smem_src)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() {
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() {
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+constexpr uint32_t kSpinLimit = 1u << 22;  // polls before a device-side wait gives up
 
 // Order-preserving map from fp32 bit patterns to unsigned integers: a larger key is a
 // larger score; negatives sort below non-negatives and -0 below +0.

@@ -2,96 +2,78 @@
 // dst[p][j][:] = src[p][keep[j]][:] for every K and V plane, all planes in one launch.
 //
 // Pure data movement, bound by HBM bandwidth (each moved row is read once and written
-// once).  A "worker" is one warp that owns a ring of shared-memory stages and walks the
-// moved rows of one plane front to back, 32 rows (one chunk) at a time:
+// once).  A "worker" is one warp that owns a ring of shared-memory stages and walks a run
+// of moved rows of one plane front to back, 32 rows (one chunk) at a time:
 //   - the lanes issue TMA bulk loads global -> shared, one per run of consecutive source
 //     rows, completing on the stage's mbarrier;
 //   - a few chunks later lane 0 waits for that mbarrier and issues ONE bulk store
 //     shared -> global for the whole chunk (destination rows are contiguous).
+// The ring keeps streaming across the boundaries of the worker's work units.
+//
 // In place (dst == src) this order is race free: the keep list is strictly ascending with
-// keep[j] >= j, so a chunk's sources lie at or behind its own first destination row.
-// A chunk is stored only after its loads and those of all earlier chunks have landed,
-// and later chunks only read rows behind everything stored so far.  Planes are
-// independent, so the ring keeps streaming across plane boundaries.
+// keep[j] >= j, so a chunk's sources lie at or behind its own first destination row.  A
+// chunk is stored only after its loads and those of all earlier chunks of the plane have
+// landed, and later chunks only read rows behind everything stored so far.
+//
+// To fill all SMs evenly, the moved rows of a plane are cut into `split` segments that
+// different workers take (segment-major order, so a plane's earlier segments are handed
+// out long before its later ones).  A segment may store only after every earlier segment
+// of its plane has landed all its loads; that is tracked by one progress word per plane
+// (epoch * 64 + finished segments) written with release and polled with acquire, with an
+// iteration limit.  All workers are resident at once (one CTA per SM at most), and a
+// worker only ever waits for a unit that precedes its own in the hand-out order, so the
+// waits cannot form a cycle.
 #include "common.cuh"
 
 namespace sirllm {
 
 namespace {
 
-constexpr int kChunkRows = 32;    // rows per chunk = one per lane
-constexpr int kStoreSlack = 2;    // bulk stores that may still be reading shared memory
+constexpr int kChunkRows = 32;  // rows per chunk = one per lane
+constexpr int kStoreSlack = 1;  // bulk stores that may still be reading shared memory
 constexpr int kMaxStages = 12;
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kMaxSplit = 32;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
-                 "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes,
-                                          uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
-            "r"(smem_u32(smem_dst)),
-        "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
-        : "memory");
-}
-__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst),
-                 "r"(smem_u32(smem_src)), "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() {
-    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void bulk_wait_all() {
-    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-}
-
-struct WorkerRing {
-    uint64_t* full;      // [stages] mbarriers
-    char** st_dst;       // [stages] destination of the chunk held by the stage
-    uint32_t* st_bytes;  // [stages]
-    char* buf;           // stages * stage_bytes
+struct StageInfo {
+    char* dst;           // destination of the chunk held by the stage
+    int32_t* flag;       // progress word of the chunk's plane
+    uint32_t bytes;
+    uint32_t wait_val;   // != 0: the store must wait until *flag == wait_val
+    uint32_t signal_val; // != 0: once the chunk's loads have landed set *flag = signal_val
+    uint32_t pad;
 };
 
-// Lane 0 waits for the loads of chunk c and stores it.  Returns false on timeout.
-__device__ __forceinline__ bool store_chunk(const WorkerRing& ring, int64_t c, int stages,
-                                            uint32_t stage_bytes, int lane) {
+__device__ __forceinline__ uint32_t ld_acquire(const int32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(int32_t* p, uint32_t v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// Lane 0 waits for the loads of chunk c, honours the plane's progress word and stores the
+// chunk.  Returns false (to all lanes) if a wait ran out.
+__device__ __forceinline__ bool store_chunk(uint64_t* full, StageInfo* info, char* buf, int64_t c,
+                                            int stages, uint32_t stage_bytes, int lane) {
     bool ok = true;
     if (lane == 0) {
         const int stage = (int)(c % stages);
         const uint32_t parity = (uint32_t)((c / stages) & 1);
-        uint32_t spins = 0;
-        while (!mbar_try_wait(&ring.full[stage], parity)) {
-            if (++spins > kSpinLimit) {
-                ok = false;
-                break;
+        ok = mbar_wait_bounded(&full[stage], parity, kSpinLimit);
+        const StageInfo si = info[stage];
+        if (ok && si.wait_val != 0) {
+            uint32_t spins = 0;
+            while (ld_acquire(si.flag) != si.wait_val) {
+                if (++spins > kSpinLimit) {
+                    ok = false;
+                    break;
+                }
             }
         }
         if (ok) {
-            bulk_store(ring.st_dst[stage], ring.buf + (size_t)stage * stage_bytes,
-                       ring.st_bytes[stage]);
+            if (si.signal_val != 0) st_release(si.flag, si.signal_val);
+            bulk_store(si.dst, buf + (size_t)stage * stage_bytes, si.bytes);
             bulk_commit();
         }
     }
@@ -99,63 +81,78 @@ __device__ __forceinline__ bool store_chunk(const WorkerRing& ring, int64_t c, i
 }
 
 __global__ void __launch_bounds__(256, 1)
-compact_kernel(const CompactParams p, const int stages, const int n_units) {
+compact_kernel(const CompactParams p, const int stages, const int units_base, const int split) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int n_workers = blockDim.x >> 5;
     const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t stage_bytes = (uint32_t)kChunkRows * (uint32_t)p.row_bytes;
 
-    // shared memory: [workers][stages] mbarriers, destinations, sizes; then the rings
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw);
-    char** dsts = reinterpret_cast<char**>(bars + n_workers * kMaxStages);
-    uint32_t* sizes = reinterpret_cast<uint32_t*>(dsts + n_workers * kMaxStages);
-    size_t header = (size_t)n_workers * kMaxStages * (8 + 8 + 4);
+    // shared memory: [workers][kMaxStages] mbarriers and stage records, then the rings
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw) + wid * kMaxStages;
+    StageInfo* info =
+        reinterpret_cast<StageInfo*>(smem_raw + (size_t)n_workers * kMaxStages * 8) + wid * kMaxStages;
+    size_t header = (size_t)n_workers * kMaxStages * (8 + sizeof(StageInfo));
     header = (header + 127) & ~(size_t)127;
-    WorkerRing ring;
-    ring.full = bars + wid * kMaxStages;
-    ring.st_dst = dsts + wid * kMaxStages;
-    ring.st_bytes = sizes + wid * kMaxStages;
-    ring.buf = reinterpret_cast<char*>(smem_raw) + header + (size_t)wid * stages * stage_bytes;
+    char* buf = reinterpret_cast<char*>(smem_raw) + header + (size_t)wid * stages * stage_bytes;
 
     if (lane == 0) {
-        for (int i = 0; i < stages; ++i) mbar_init(&ring.full[i], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        for (int i = 0; i < stages; ++i) mbar_init(&full[i], 1);
+        mbar_init_fence();
     }
     __syncwarp();
-    grid_dependency_wait();  // the keep lists of the selection kernel
+    grid_dependency_wait();  // the keep lists (and the epoch) of the preceding kernel
 
+    const uint32_t epoch_base = ((uint32_t)*p.epoch << 6) | 0x80000000u;  // never 0
     const int lead = stages - 1 - kStoreSlack;  // chunks whose loads run ahead of the stores
     const int64_t g = (int64_t)blockIdx.x * n_workers + wid;
     const int64_t G = (int64_t)gridDim.x * n_workers;
+    const int64_t n_units = (int64_t)units_base * split;
     int64_t it = 0;      // chunks whose loads were issued
     int64_t stored = 0;  // chunks whose store was issued
     bool alive = true;
 
     for (int64_t u = g; u < n_units && alive; u += G) {
-        const int tensor = (int)(u / p.planes_per_tensor);
-        const int64_t plane = u - (int64_t)tensor * p.planes_per_tensor;
+        const int h = (int)(u / units_base);  // segment of the plane's moved rows
+        const int r = (int)(u - (int64_t)h * units_base);
+        const int tensor = (int)(r / p.planes_per_tensor);
+        const int64_t plane = r - (int64_t)tensor * p.planes_per_tensor;
         const int s = (int)(plane / p.planes_per_stream);
         const int n = min(max(p.n_keep[s], 0), p.keep_stride);
         int f = p.first_moved[s];
         if (f < 0) continue;  // keep list rejected
         if (!p.in_place) f = 0;
+        if (f >= n) continue;
+        const int total_chunks = (n - f + kChunkRows - 1) / kChunkRows;
+        const int per_seg = (total_chunks + split - 1) / split;
+        const int n_seg = (total_chunks + per_seg - 1) / per_seg;  // non-empty segments
+        if (h >= n_seg) continue;
+        const int c_begin = h * per_seg, c_end = min(total_chunks, c_begin + per_seg);
+        const int j_begin = f + c_begin * kChunkRows, j_end = min(n, f + c_end * kChunkRows);
+
         const char* src = (tensor ? p.src[1] : p.src[0]) + (size_t)plane * p.capacity * p.row_bytes;
         char* dst = (tensor ? p.dst[1] : p.dst[0]) + (size_t)plane * p.capacity * p.row_bytes;
         const int32_t* keep = p.keep_idx + (size_t)s * p.keep_stride;
+        const bool chained = p.in_place && n_seg > 1;
 
-        int kj_next = f + lane < n ? keep[f + lane] : -2;  // source rows of the first chunk
-        for (int j0 = f; j0 < n && alive; j0 += kChunkRows) {
-            const int nrows = min(kChunkRows, n - j0);
+        int kj_next = j_begin + lane < j_end ? keep[j_begin + lane] : -2;  // first chunk's sources
+        for (int j0 = j_begin; j0 < j_end && alive; j0 += kChunkRows) {
+            const int nrows = min(kChunkRows, j_end - j0);
             const int stage = (int)(it % stages);
             const int kj = kj_next;
             // fetch the next chunk's source rows now; they are needed one trip later
-            kj_next = j0 + kChunkRows + lane < n ? keep[j0 + kChunkRows + lane] : -2;
+            kj_next = j0 + kChunkRows + lane < j_end ? keep[j0 + kChunkRows + lane] : -2;
             if (lane == 0) {
                 if (it >= stages) bulk_wait_read<kStoreSlack>();  // the stage's last store has left
-                ring.st_dst[stage] = dst + (size_t)j0 * p.row_bytes;
-                ring.st_bytes[stage] = (uint32_t)nrows * p.row_bytes;
-                mbar_expect_tx(&ring.full[stage], (uint32_t)nrows * p.row_bytes);
+                StageInfo si;
+                si.dst = dst + (size_t)j0 * p.row_bytes;
+                si.flag = p.plane_flags + r;
+                si.bytes = (uint32_t)nrows * p.row_bytes;
+                si.wait_val = (chained && h > 0 && j0 == j_begin) ? epoch_base + h : 0u;
+                si.signal_val =
+                    (chained && h + 1 < n_seg && j0 + kChunkRows >= j_end) ? epoch_base + h + 1 : 0u;
+                si.pad = 0;
+                info[stage] = si;
+                mbar_expect_tx(&full[stage], si.bytes);
             }
             __syncwarp();
             // one bulk load per run of consecutive source rows
@@ -165,19 +162,19 @@ compact_kernel(const CompactParams p, const int stages, const int n_units) {
             if (head) {
                 const uint32_t later = lane == 31 ? 0u : (heads & ~((2u << lane) - 1u));
                 const int next = later ? __ffs(later) - 1 : nrows;
-                bulk_load(ring.buf + (size_t)stage * stage_bytes + (size_t)lane * p.row_bytes,
+                bulk_load(buf + (size_t)stage * stage_bytes + (size_t)lane * p.row_bytes,
                           src + (size_t)kj * p.row_bytes, (uint32_t)(next - lane) * p.row_bytes,
-                          &ring.full[stage]);
+                          &full[stage]);
             }
             ++it;
             if (it - stored > lead) {
-                alive = store_chunk(ring, stored, stages, stage_bytes, lane);
+                alive = store_chunk(full, info, buf, stored, stages, stage_bytes, lane);
                 ++stored;
             }
         }
     }
     while (alive && stored < it) {
-        alive = store_chunk(ring, stored, stages, stage_bytes, lane);
+        alive = store_chunk(full, info, buf, stored, stages, stage_bytes, lane);
         ++stored;
     }
     if (lane == 0) {
@@ -195,6 +192,7 @@ __global__ void compact_plan_kernel(const CompactParams p, int32_t* __restrict__
     if (threadIdx.x == 0) {
         sh_first = n;
         sh_bad = (p.n_keep[s] < 0 || p.n_keep[s] > p.keep_stride) ? 1 : 0;
+        if (s == 0) *p.epoch += 1;  // a new compaction follows
     }
     __syncthreads();
     for (int j = threadIdx.x; j < n; j += blockDim.x) {
@@ -234,8 +232,8 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     }
     const int64_t units64 = (int64_t)n_tensors * p.planes_per_tensor;
     if (units64 == 0) return cudaSuccess;
-    if (units64 > 0x7FFFFFFF) return cudaErrorInvalidValue;
-    const int n_units = (int)units64;
+    if (units64 > 0x3FFFFFFF) return cudaErrorInvalidValue;
+    const int units_base = (int)units64;
 
     int dev = 0, n_sm = 0, smem_max = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -247,17 +245,35 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
 
     // ring geometry: as many workers per SM as fit with at least 6 stages each (at most 8)
     const size_t stage_bytes = (size_t)kChunkRows * p.row_bytes;
-    const size_t budget = (size_t)smem_max - 1024;
+    const size_t budget = (size_t)smem_max - 2048;
     int workers = 4, stages = 6;
     while (workers > 1 && (size_t)workers * stages * stage_bytes > budget) --workers;
     while (stages > 4 && (size_t)workers * stages * stage_bytes > budget) --stages;
     if ((size_t)workers * stages * stage_bytes > budget) return cudaErrorInvalidValue;
     while (stages < 8 && (size_t)workers * (stages + 1) * stage_bytes <= budget) ++stages;
-    size_t header = (size_t)workers * kMaxStages * (8 + 8 + 4);
+    size_t header = (size_t)workers * kMaxStages * (8 + sizeof(StageInfo));
     header = (header + 127) & ~(size_t)127;
     const size_t smem = header + (size_t)workers * stages * stage_bytes;
     e = cudaFuncSetAttribute(compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
+
+    // one CTA per SM at most (all workers resident); cut planes into segments so that the
+    // units spread evenly over the workers: fewest idle worker-rounds, then fewest segments
+    const int64_t slots = (int64_t)n_sm * workers;
+    int split = 1;
+    if (units_base < 8 * slots) {
+        double best = -1.0;
+        for (int h = 1; h <= kMaxSplit; ++h) {
+            const int64_t units = (int64_t)units_base * h;
+            const int64_t rounds = (units + slots - 1) / slots;
+            const double eff = (double)units / (double)(rounds * slots);
+            if (eff > best + 0.02) {
+                best = eff;
+                split = h;
+            }
+        }
+    }
+    const int64_t n_units = (int64_t)units_base * split;
     const int grid = (int)((n_units + workers - 1) / workers < n_sm ? (n_units + workers - 1) / workers
                                                                     : n_sm);
     cudaLaunchConfig_t cfg = {};
@@ -270,7 +286,7 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, compact_kernel, q, stages, n_units);
+    return cudaLaunchKernelEx(&cfg, compact_kernel, q, stages, units_base, split);
 }
 
 }  // namespace sirllm

@@ -62,6 +62,7 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     int32_t* keep = p.keep_idx + (size_t)s * p.threshold;
     grid_launch_dependents();
     grid_dependency_wait();  // the scorer's appended scores
+    if (blockIdx.x == 0 && tid == 0) *p.epoch += 1;  // a new compaction follows
 
     const int l0 = p.live_len[s];
     int T = 0;
