@@ -33,6 +33,7 @@ constexpr int kChunkRows = 32;  // rows per chunk = one per lane
 constexpr int kStoreSlack = 1;  // bulk stores that may still be reading shared memory
 constexpr int kMaxStages = 12;
 constexpr int kMaxSplit = 32;
+constexpr int kIdxAhead = 4;  // chunks whose source indices are fetched ahead
 
 struct StageInfo {
     char* dst;           // destination of the chunk held by the stage
@@ -134,43 +135,62 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
         const int32_t* keep = p.keep_idx + (size_t)s * p.keep_stride;
         const bool chained = p.in_place && n_seg > 1;
 
-        int kj_next = j_begin + lane < j_end ? keep[j_begin + lane] : -2;  // first chunk's sources
-        for (int j0 = j_begin; j0 < j_end && alive; j0 += kChunkRows) {
-            const int nrows = min(kChunkRows, j_end - j0);
-            const int stage = (int)(it % stages);
-            const int kj = kj_next;
-            // fetch the next chunk's source rows now; they are needed one trip later
-            kj_next = j0 + kChunkRows + lane < j_end ? keep[j0 + kChunkRows + lane] : -2;
-            if (lane == 0) {
-                if (it >= stages) bulk_wait_read<kStoreSlack>();  // the stage's last store has left
-                StageInfo si;
-                si.dst = dst + (size_t)j0 * p.row_bytes;
-                si.flag = p.plane_flags + r;
-                si.bytes = (uint32_t)nrows * p.row_bytes;
-                si.wait_val = (chained && h > 0 && j0 == j_begin) ? epoch_base + h : 0u;
-                si.signal_val =
-                    (chained && h + 1 < n_seg && j0 + kChunkRows >= j_end) ? epoch_base + h + 1 : 0u;
-                si.pad = 0;
-                info[stage] = si;
-                mbar_expect_tx(&full[stage], si.bytes);
+        // source rows of the next kIdxAhead chunks, one per lane and chunk, fetched a whole
+        // group ahead so that the index loads never sit on the critical path
+        int kq[kIdxAhead];
+#pragma unroll
+        for (int q = 0; q < kIdxAhead; ++q) {
+            const int j = j_begin + q * kChunkRows + lane;
+            kq[q] = j < j_end ? keep[j] : -2;
+        }
+        for (int jg = j_begin; jg < j_end && alive; jg += kIdxAhead * kChunkRows) {
+            int kn[kIdxAhead];
+#pragma unroll
+            for (int q = 0; q < kIdxAhead; ++q) {
+                const int j = jg + (kIdxAhead + q) * kChunkRows + lane;
+                kn[q] = j < j_end ? keep[j] : -2;
             }
-            __syncwarp();
-            // one bulk load per run of consecutive source rows
-            const int prev = __shfl_up_sync(0xFFFFFFFFu, kj, 1);
-            const bool head = lane < nrows && (lane == 0 || kj != prev + 1);
-            const uint32_t heads = __ballot_sync(0xFFFFFFFFu, head);
-            if (head) {
-                const uint32_t later = lane == 31 ? 0u : (heads & ~((2u << lane) - 1u));
-                const int next = later ? __ffs(later) - 1 : nrows;
-                bulk_load(buf + (size_t)stage * stage_bytes + (size_t)lane * p.row_bytes,
-                          src + (size_t)kj * p.row_bytes, (uint32_t)(next - lane) * p.row_bytes,
-                          &full[stage]);
+#pragma unroll
+            for (int q = 0; q < kIdxAhead; ++q) {
+                const int j0 = jg + q * kChunkRows;
+                if (j0 >= j_end || !alive) break;
+                const int nrows = min(kChunkRows, j_end - j0);
+                const int stage = (int)(it % stages);
+                const int kj = kq[q];
+                if (lane == 0) {
+                    if (it >= stages) bulk_wait_read<kStoreSlack>();  // the stage's last store has left
+                    StageInfo si;
+                    si.dst = dst + (size_t)j0 * p.row_bytes;
+                    si.flag = p.plane_flags + r;
+                    si.bytes = (uint32_t)nrows * p.row_bytes;
+                    si.wait_val = (chained && h > 0 && j0 == j_begin) ? epoch_base + h : 0u;
+                    si.signal_val = (chained && h + 1 < n_seg && j0 + kChunkRows >= j_end)
+                                        ? epoch_base + h + 1
+                                        : 0u;
+                    si.pad = 0;
+                    info[stage] = si;
+                    mbar_expect_tx(&full[stage], si.bytes);
+                }
+                __syncwarp();
+                // one bulk load per run of consecutive source rows
+                const int prev = __shfl_up_sync(0xFFFFFFFFu, kj, 1);
+                const bool head = lane < nrows && (lane == 0 || kj != prev + 1);
+                const uint32_t heads = __ballot_sync(0xFFFFFFFFu, head);
+                if (head) {
+                    const uint32_t later = lane == 31 ? 0u : (heads & ~((2u << lane) - 1u));
+                    const int next = later ? __ffs(later) - 1 : nrows;
+                    bulk_load(buf + (size_t)stage * stage_bytes + (size_t)lane * p.row_bytes,
+                              src + (size_t)kj * p.row_bytes, (uint32_t)(next - lane) * p.row_bytes,
+                              &full[stage]);
+                }
+                ++it;
+                if (it - stored > lead) {
+                    alive = store_chunk(full, info, buf, stored, stages, stage_bytes, lane);
+                    ++stored;
+                }
             }
-            ++it;
-            if (it - stored > lead) {
-                alive = store_chunk(full, info, buf, stored, stages, stage_bytes, lane);
-                ++stored;
-            }
+#pragma unroll
+            for (int q = 0; q < kIdxAhead; ++q) kq[q] = kn[q];
         }
     }
     while (alive && stored < it) {
