@@ -27,8 +27,8 @@ struct WorkspaceLayout {
     int32_t n_part;  // CTAs (groups of kScoreWarpsPerCta segments) per logits row
 };
 
-constexpr int kVecPerSeg = 512;  // 16-byte vectors per segment: 8 KB of logits per warp
-constexpr int kScoreWarpsPerCta = 8;
+constexpr int kVecPerSeg = 1024;  // 16-byte vectors per segment: 16 KB of logits per warp
+constexpr int kScoreWarpsPerCta = 4;
 constexpr int kSelectThreads = 1024;
 constexpr int kRadixBits = 11;
 constexpr int kRadixBins = 1 << kRadixBits;

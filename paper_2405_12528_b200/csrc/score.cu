@@ -91,9 +91,8 @@ score_kernel(const ScoreParams p) {
     const int64_t v1 = min(v0 + (int64_t)kVecPerSeg, nvec);
     const uint32_t neg_inf = kBf16 ? 0xFF80FF80u : 0xFF800000u;
 
-    Online st;
-    for (int64_t base = v0; base < v1; base += 32 * kUnroll) {
-        uint4 x[kUnroll];
+    // software pipeline: the loads of trip i+1 are in flight while trip i is reduced
+    auto fetch = [&](int64_t base, uint4 (&x)[kUnroll]) {
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
             const int64_t idx = base + u * 32 + lane;
@@ -102,6 +101,12 @@ score_kernel(const ScoreParams p) {
             else
                 x[u] = make_uint4(neg_inf, neg_inf, neg_inf, neg_inf);
         }
+    };
+    Online st;
+    uint4 x[kUnroll], xn[kUnroll];
+    if (v0 < v1) fetch(v0, x);
+    for (int64_t base = v0; base < v1; base += 32 * kUnroll) {
+        fetch(base + 32 * kUnroll, xn);  // past the end: filled with -inf, never reduced
         if (kBf16) {
             uint32_t m2 = x[0].x;
 #pragma unroll
@@ -137,6 +142,8 @@ score_kernel(const ScoreParams p) {
                 st.add1(__uint_as_float(x[u].w));
             }
         }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) x[u] = xn[u];
     }
     // ragged ends of the row (fewer than one vector each) go to segment 0
     if (seg == 0 && lane < head + tail) {
