@@ -48,6 +48,7 @@ extern "C" {
 #define SIRLLM_ERR_BAD_CONFIG (-2) /* inconsistent or unsupported sirllm_config */
 #define SIRLLM_ERR_ALIGN (-3)      /* a pointer or stride breaks the 16-byte alignment rule */
 #define SIRLLM_ERR_CUDA (-4)       /* a CUDA runtime call failed; see sirllm_last_cuda_error() */
+#define SIRLLM_ERR_TOO_LARGE (-5)  /* the problem exceeds a fixed limit of the entry point */
 
 /* bits of the device status word */
 #define SIRLLM_STATUS_TOKEN_RANGE 1 /* a token id outside [0, vocab) other than -1; scored 0 */
@@ -103,6 +104,37 @@ int sirllm_workspace_init(const sirllm_config *cfg, void *ws, void *cuda_stream)
  */
 int sirllm_score(const sirllm_config *cfg, const void *logits, const int32_t *token_ids,
                  const int32_t *n_new, float *out_entropy, void *ws, void *cuda_stream);
+
+/*
+ * sirllm_score for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this is a packaging variant of the same kernel.)
+ *
+ * Who needs it: code that runs where every device allocation belongs to someone else - a
+ * plugin or custom-op slot inside a host framework that passes fixed inputs and outputs and
+ * no scratch - or that must not call the allocator at that moment because an allocation
+ * can synchronise the whole device or fail when memory is tight.  Such a caller has no
+ * place to put the workspace sirllm_score wants, so this entry point takes none: its
+ * scratch (the per-row tickets and per-CTA partial sums, 590080 bytes) is a fixed array
+ * inside the library image.  It calls no cudaMalloc / cudaFree and no allocating routine.
+ *
+ * Same arguments and result as sirllm_score (scores are bit-identical), except:
+ *   status   int32 device word that receives SIRLLM_STATUS_* bits (OR-ed in; the caller
+ *            zeroes it), or NULL to drop them
+ *   limits   n_streams * max_new <= 16384 rows, and rows * ceil(vocab / 32768 [bf16] or
+ *            16384 [fp32]) <= 65536; beyond that SIRLLM_ERR_TOO_LARGE is returned and
+ *            nothing runs
+ * Things to know:
+ *   - every GPU that loads the library holds the array until the process exits;
+ *   - the first call on each device looks up the array's address on that device (the
+ *     device must be current, as for any call here); make that first call before any
+ *     stream capture starts;
+ *   - all calls on a device share the array: each call clears the part that must start
+ *     at zero with a memset on `cuda_stream`, so calls ordered on one stream are safe, but
+ *     two calls that can overlap on the GPU (different streams, no dependency) race.
+ */
+int sirllm_score_static(const sirllm_config *cfg, const void *logits, const int32_t *token_ids,
+                        const int32_t *n_new, float *out_entropy, int32_t *status,
+                        void *cuda_stream);
 
 /*
  * Memory decay and selection (Section 3.3: E = E x eta_decay, Id_entropy = Top_k(E);

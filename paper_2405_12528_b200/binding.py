@@ -17,11 +17,12 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libsirllm.so")
 
 F32, BF16, F16 = 0, 1, 2
-OK, ERR_NULL, ERR_BAD_CONFIG, ERR_ALIGN, ERR_CUDA = 0, -1, -2, -3, -4
+OK, ERR_NULL, ERR_BAD_CONFIG, ERR_ALIGN, ERR_CUDA, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5
 STATUS_TOKEN_RANGE, STATUS_OVERFLOW, STATUS_TIMEOUT, STATUS_BAD_KEEP = 1, 2, 4, 8
 MAX_CAPACITY = 49152
 
-EXPORTS = ["sirllm_workspace_bytes", "sirllm_workspace_init", "sirllm_score", "sirllm_decay_select",
+EXPORTS = ["sirllm_workspace_bytes", "sirllm_workspace_init", "sirllm_score", "sirllm_score_static",
+           "sirllm_decay_select",
            "sirllm_compact_kv", "sirllm_step", "sirllm_step_phases", "sirllm_step_host",
            "sirllm_status", "sirllm_strerror",
            "sirllm_last_cuda_error"]
@@ -85,6 +86,8 @@ def lib():
         L.sirllm_workspace_init.argtypes = [cfgp, vp, vp]
         L.sirllm_score.restype = ctypes.c_int
         L.sirllm_score.argtypes = [cfgp, vp, vp, vp, vp, vp, vp]
+        L.sirllm_score_static.restype = ctypes.c_int
+        L.sirllm_score_static.argtypes = [cfgp, vp, vp, vp, vp, vp, vp]
         L.sirllm_decay_select.restype = ctypes.c_int
         L.sirllm_decay_select.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, i32, vp, vp]
         L.sirllm_compact_kv.restype = ctypes.c_int
@@ -165,6 +168,17 @@ def sirllm_score(cfg: Config, logits, token_ids, n_new, out_entropy, ws) -> None
                               _dev(n_new, torch.int32, "n_new"),
                               _dev(out_entropy, torch.float32, "out_entropy"),
                               _dev(ws, torch.uint8, "ws"), _stream()))
+
+
+def sirllm_score_static(cfg: Config, logits, token_ids, n_new, out_entropy, status=None) -> None:
+    """``sirllm_score`` without a workspace: for callers that cannot allocate device memory
+    (the scratch is a fixed array inside the library; at most 16384 logits rows per call,
+    and calls that overlap on the GPU race).  ``status``: optional int32 device word."""
+    _check(lib().sirllm_score_static(ctypes.byref(cfg), _logits_ptr(cfg, logits),
+                                     _dev(token_ids, torch.int32, "token_ids"),
+                                     _dev(n_new, torch.int32, "n_new"),
+                                     _dev(out_entropy, torch.float32, "out_entropy"),
+                                     _dev(status, torch.int32, "status"), _stream()))
 
 
 def sirllm_decay_select(cfg: Config, scores, serial, live_len, decay, keep_idx, n_keep,

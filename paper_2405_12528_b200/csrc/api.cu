@@ -358,6 +358,7 @@ const char* sirllm_strerror(int code) {
         case SIRLLM_ERR_BAD_CONFIG: return "inconsistent or unsupported configuration";
         case SIRLLM_ERR_ALIGN: return "pointer or stride not aligned as required";
         case SIRLLM_ERR_CUDA: return "CUDA runtime error (see sirllm_last_cuda_error)";
+        case SIRLLM_ERR_TOO_LARGE: return "problem larger than the fixed limit of this entry point";
         default: return "unknown error code";
     }
 }

@@ -228,3 +228,89 @@ cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
 }
 
 }  // namespace sirllm
+
+// ---------------------------------------------------------------------------------------------
+// sirllm_score_static: scoring for callers that cannot allocate device memory.
+//
+// sirllm_score needs a caller-allocated workspace for its tickets and per-CTA partial pairs.
+// Some callers cannot provide one: code that runs inside a host framework which owns every
+// allocation and hands out no scratch (a plugin or custom-op slot with fixed inputs and
+// outputs), or code that must not touch the allocator at that point of the program (an
+// allocation may synchronise the device or fail under memory pressure).  For them the same
+// kernel runs on a scratch area that is part of the library image: a file-scope device
+// array.  Every GPU that loads the library holds these kSsBytes bytes until the process
+// exits, every call on a device shares them (so two calls that overlap on the GPU race),
+// and the array keeps whatever the last call left in it, so each call first clears the part
+// that has to start at zero.
+namespace {
+
+constexpr int64_t kSsMaxRows = 16384;    // logits rows (n_streams * max_new) per call
+constexpr int64_t kSsMaxPairs = 65536;   // rows * CTAs per row
+constexpr size_t kSsStatusOff = 0;                              // int32 status word
+constexpr size_t kSsTicketsOff = 256;                           // int32 [kSsMaxRows]
+constexpr size_t kSsPairsOff = kSsTicketsOff + kSsMaxRows * 4;  // float2 [kSsMaxPairs]
+constexpr size_t kSsBytes = kSsPairsOff + kSsMaxPairs * 8;      // 590080 bytes
+
+static __device__ __align__(256) unsigned char g_score_scratch[kSsBytes];
+
+// In host code `g_score_scratch` is only a handle of the symbol, not a device address: the
+// address each device gave the array is looked up once per device and remembered here.
+constexpr int kSsMaxDevices = 64;
+void* g_scratch_addr[kSsMaxDevices] = {};
+
+cudaError_t scratch_address(void** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kSsMaxDevices) return cudaErrorInvalidDevice;
+    void* addr = __atomic_load_n(&g_scratch_addr[dev], __ATOMIC_ACQUIRE);
+    if (addr == nullptr) {
+        e = cudaGetSymbolAddress(&addr, g_score_scratch);  // of the CURRENT device
+        if (e != cudaSuccess) return e;
+        __atomic_store_n(&g_scratch_addr[dev], addr, __ATOMIC_RELEASE);
+    }
+    *out = addr;
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int sirllm_score_static(const sirllm_config* cfg, const void* logits,
+                                   const int32_t* token_ids, const int32_t* n_new,
+                                   float* out_entropy, int32_t* status, void* cuda_stream) {
+    using namespace sirllm;
+    int rc = validate_config(cfg);
+    if (rc != SIRLLM_OK) return rc;
+    if (!logits || !token_ids || !out_entropy) return SIRLLM_ERR_NULL;
+    if (((uintptr_t)logits % (size_t)logits_elem_bytes(cfg->logits_dtype)) != 0) return SIRLLM_ERR_ALIGN;
+    const WorkspaceLayout L = workspace_layout(*cfg);
+    const int64_t rows = (int64_t)cfg->n_streams * cfg->max_new;
+    if (rows > kSsMaxRows || rows * L.n_part > kSsMaxPairs) return SIRLLM_ERR_TOO_LARGE;
+    if (rows == 0) return SIRLLM_OK;
+    void* base = nullptr;
+    cudaError_t e = scratch_address(&base);
+    if (e != cudaSuccess) return SIRLLM_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // status word and tickets must start at zero; the pairs are written before they are read
+    e = cudaMemsetAsync(base, 0, kSsTicketsOff + (size_t)rows * 4, st);
+    if (e != cudaSuccess) return SIRLLM_ERR_CUDA;
+    ScoreParams sp;
+    sp.logits = logits;
+    sp.token_ids = token_ids;
+    sp.n_new = n_new;
+    sp.partials = (float2*)((char*)base + kSsPairsOff);
+    sp.tickets = (int32_t*)((char*)base + kSsTicketsOff);
+    sp.status = status ? status : (int32_t*)((char*)base + kSsStatusOff);
+    sp.out_entropy = out_entropy;
+    sp.scores = nullptr;
+    sp.live_len = nullptr;
+    sp.vocab = cfg->vocab;
+    sp.row_stride = cfg->logits_row_stride;
+    sp.n_streams = cfg->n_streams;
+    sp.max_new = cfg->max_new;
+    sp.n_part = L.n_part;
+    sp.logits_dtype = cfg->logits_dtype;
+    sp.capacity = cfg->capacity;
+    e = launch_score(sp, st);
+    return e == cudaSuccess ? SIRLLM_OK : SIRLLM_ERR_CUDA;
+}
