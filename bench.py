@@ -30,6 +30,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+from paper_2405_12528_b200 import sharding  # noqa: E402
 from paper_2405_12528_b200 import workloads as wl  # noqa: E402
 
 METRIC = "tokens/s through entropy+decay+top-k eviction; KV compaction GB/s vs HBM peak"
@@ -102,16 +103,18 @@ class ClockSampler:
 class Pass:
     """Device state of one rank and the calls of one round."""
 
-    def __init__(self, w: wl.Workload, seed: int, dev: str):
+    def __init__(self, w: wl.Workload, seed: int, dev: str, stream_ids=None):
         from paper_2405_12528_b200 import binding as B
         self.B, self.w, self.seed, self.dev = B, w, seed, dev
+        # global ids of the streams this rank hosts: they key the seeded inputs
+        self.sid = list(stream_ids) if stream_ids is not None else list(range(w.n_streams))
         self.cfg = B.config_from_workload(w)
         S, P, C, D, M = w.n_streams, w.planes_per_stream, w.capacity, w.head_dim, w.new_tokens
         self.ws = B.new_workspace(self.cfg, dev)
         self.scores = torch.zeros(S, C, dtype=torch.float32, device=dev)
         self.serial = torch.full((S, C), -1, dtype=torch.int64, device=dev)
         self.live_len = torch.zeros(S, dtype=torch.int32, device=dev)
-        self.decay = wl.stream_decay(w, seed).to(dev)
+        self.decay = wl.stream_decay(w.scaled(n_streams=max(self.sid) + 1), seed)[self.sid].to(dev)
         self.keep_idx = torch.zeros(S, self.cfg.threshold, dtype=torch.int32, device=dev)
         self.n_keep = torch.zeros(S, dtype=torch.int32, device=dev)
         self.new_entropy = torch.zeros(S * M, dtype=torch.float32, device=dev)
@@ -124,8 +127,8 @@ class Pass:
             lg = torch.empty(S * M, w.vocab, dtype=w.torch_logits_dtype, device=dev)
             ids = torch.empty(S * M, dtype=torch.int32, device=dev)
             for s in range(S):
-                wl.make_logits(w, seed, s, r, M, dev, bias, out=lg[s * M:(s + 1) * M])
-                ids[s * M:(s + 1) * M] = wl.make_token_ids(w, seed, s, r, M, dev)
+                wl.make_logits(w, seed, self.sid[s], r, M, dev, bias, out=lg[s * M:(s + 1) * M])
+                ids[s * M:(s + 1) * M] = wl.make_token_ids(w, seed, self.sid[s], r, M, dev)
             self.pool.append((lg, ids))
         self.next_serial = 0
         self.round = 0
@@ -139,8 +142,8 @@ class Pass:
         for s in range(w.n_streams):
             l = lens[s]
             self.serial[s, l:l + T] = serials
-            self.k[s, :, l:l + T] = wl.make_kv_rows(w, self.seed, "k", s, serials, device=self.dev)
-            self.v[s, :, l:l + T] = wl.make_kv_rows(w, self.seed, "v", s, serials, device=self.dev)
+            self.k[s, :, l:l + T] = wl.make_kv_rows(w, self.seed, "k", self.sid[s], serials, device=self.dev)
+            self.v[s, :, l:l + T] = wl.make_kv_rows(w, self.seed, "v", self.sid[s], serials, device=self.dev)
         self.next_serial += T
 
     def step(self, events=None):
@@ -192,7 +195,7 @@ def run_ours(args, rank, world, local_rank):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(dev))
-    p = Pass(w, seed=rank, dev=dev)
+    p = Pass(w, seed=0, dev=dev, stream_ids=sharding.owned_streams(w.n_streams, rank))
     p.prime()
 
     cpu_baseline = None
@@ -215,11 +218,7 @@ def run_ours(args, rank, world, local_rank):
             p.step()
         t1.record()
         sync()
-    ms_total = t0.elapsed_time(t1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t[0])
+    ms_total = sharding.max_over_ranks(t0.elapsed_time(t1), dev)
     assert B.sirllm_status(p.ws) == 0
     ms_step = ms_total / args.steps
     tokens = world * w.n_streams * w.new_tokens
@@ -285,8 +284,8 @@ def run_e2e(p: Pass, args, dist, world):
     h_k = torch.empty(S, P, M, D, dtype=w.torch_kv_dtype).pin_memory()
     h_v = torch.empty(S, P, M, D, dtype=w.torch_kv_dtype).pin_memory()
     for s in range(S):
-        h_k[s] = wl.make_kv_rows(w, p.seed, "k", s, serials, device=p.dev).cpu()
-        h_v[s] = wl.make_kv_rows(w, p.seed, "v", s, serials, device=p.dev).cpu()
+        h_k[s] = wl.make_kv_rows(w, p.seed, "k", p.sid[s], serials, device=p.dev).cpu()
+        h_v[s] = wl.make_kv_rows(w, p.seed, "v", p.sid[s], serials, device=p.dev).cpu()
     h_n_new = torch.full((S,), M, dtype=torch.int32).pin_memory()
     h_len = p.live_len.cpu().pin_memory()
     h_keep = torch.zeros(S, cfg.threshold, dtype=torch.int32).pin_memory()
@@ -314,11 +313,7 @@ def run_e2e(p: Pass, args, dist, world):
     for i in range(n):
         one(i)
     torch.cuda.synchronize()
-    dt = time.perf_counter() - t0
-    if dist is not None:
-        t = torch.tensor([dt], device=p.dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dt = float(t[0])
+    dt = sharding.max_over_ranks(time.perf_counter() - t0, p.dev)
     return {"value": round(world * S * M * n / dt, 1), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": round(dt / n * 1e3, 3), "steps": n,
             "call": "sirllm_step_host"}

@@ -1,0 +1,79 @@
+"""World-size-2 run of the multi-GPU plumbing on CPU (gloo): streams shard across ranks with
+no data-path collective; only timings and counts are reduced."""
+import os
+import socket
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import oracle
+from paper_2405_12528_b200 import sharding
+from paper_2405_12528_b200 import workloads as wl
+
+
+def test_stream_ownership_is_a_partition():
+    for world in (1, 2, 3, 8):
+        ids = [i for r in range(world) for i in sharding.owned_streams(5, r)]
+        assert ids == list(range(5 * world))
+        for total in (1, 7, 64):
+            parts = [sharding.split_streams(total, world, r) for r in range(world)]
+            assert [i for p in parts for i in p] == list(range(total))
+            assert max(len(p) for p in parts) - min(len(p) for p in parts) <= 1
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _one_round_on_the_oracle(w, stream_id):
+    """One evicting round of one stream, computed by the oracle (stand-in for a GPU)."""
+    st = oracle.Stream(w.capacity, w.n_sink, w.n_recent, w.budget, w.threshold, w.decay)
+    logits = wl.make_logits(w, 0, stream_id, 0)
+    ids = wl.make_token_ids(w, 0, stream_id, 0)
+    keep = st.step(oracle.score(logits, ids))
+    return keep
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        w = wl.WORKLOADS["tiny"].scaled(new_tokens=96, budget=64, n_recent=16, vocab=997, capacity=128)
+        mine = sharding.owned_streams(2, rank)
+        digests = []
+        for sid in mine:                                    # no communication on the data path
+            keep = _one_round_on_the_oracle(w, sid)
+            digests.append(int(keep.long().sum()))
+        gathered = [None] * world
+        dist.all_gather_object(gathered, (list(mine), digests))
+        slowest = sharding.max_over_ranks(1.5 * (rank + 1))
+        tokens = sharding.sum_over_ranks(len(mine) * w.new_tokens)
+        out.put((rank, gathered, slowest, tokens))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_shard_streams_and_reduce_only_bookkeeping():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    w = wl.WORKLOADS["tiny"].scaled(new_tokens=96, budget=64, n_recent=16, vocab=997, capacity=128)
+    single = [int(_one_round_on_the_oracle(w, sid).long().sum()) for sid in range(4)]
+    for rank, gathered, slowest, tokens in results:
+        ids = [i for owned, _ in gathered for i in owned]
+        got = [d for _, dig in gathered for d in dig]
+        assert ids == [0, 1, 2, 3]                      # every stream owned exactly once
+        assert got == single                            # sharded result == single-process result
+        assert len(set(single)) > 1                     # and the streams really differ
+        assert slowest == 3.0                           # max over ranks
+        assert tokens == 4 * 96                         # whole-job count
