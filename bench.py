@@ -39,6 +39,29 @@ DEFAULT_WORKLOAD = "llama3_8b"      # the shape the 70 %-of-HBM target is quoted
 FALLBACK_HBM_GBS = 6650.0
 
 
+# DRAM traffic of the dominant kernel from one ncu capture (profiles/compact_kernel_*.md):
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch on the small profiling case.
+# Traffic grows in proportion to the moved bytes, so it is scaled to the timed launch; it
+# is reported only while the kernel's sources are the ones the counters were taken on.
+NCU_CAPTURE = {"kernel": "compact_kernel", "workload": "llama3_8b_quarter",
+               "dram_bytes": 267954688 + 214801920, "algorithmic_bytes": 2 * 2044 * 256 * 512,
+               "sources": {"paper_2405_12528_b200/csrc/compact.cu": "5a73a5c0abc81843c030398e7e68774a28b94481",
+                           "paper_2405_12528_b200/csrc/common.cuh": "2d7831351ca583eff4dd5eeda078a670e52ce9cd"}}
+
+
+def ncu_traffic(bytes_per_launch):
+    import hashlib
+    for rel, want in NCU_CAPTURE["sources"].items():
+        try:
+            with open(os.path.join(ROOT, rel), "rb") as fh:
+                b = fh.read()
+        except OSError:
+            return None
+        if hashlib.sha1(b"blob %d\0" % len(b) + b).hexdigest() != want:
+            return None          # the kernel changed since the counters were taken
+    return round(NCU_CAPTURE["dram_bytes"] * bytes_per_launch / NCU_CAPTURE["algorithmic_bytes"])
+
+
 def measured_hbm_peak():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
@@ -239,7 +262,8 @@ def run_ours(args, rank, world, local_rank):
     compact_gbs = by["compact"] / (phase_ms[2] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "compact_kernel", "achieved": round(compact_gbs, 1),
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                "frac": round(compact_gbs / peak, 4), "traffic": None,
+                "frac": round(compact_gbs / peak, 4),
+                "traffic": ncu_traffic(by["compact"]) if w.row_bytes == 256 else None,
                 "bytes_per_launch": by["compact"], "ms_per_launch": round(phase_ms[2], 4),
                 "moved_rows_per_round": mean_moved,
                 "phases_ms": {"score": round(phase_ms[0], 4), "select": round(phase_ms[1], 4),
