@@ -40,6 +40,8 @@ def lib():
         L.oracle_token_entropy.argtypes = [vp, ctypes.c_int, i64, i32, vp]
         L.oracle_score.restype = ctypes.c_int
         L.oracle_score.argtypes = [vp, ctypes.c_int, i64, i64, i64, vp, vp]
+        L.oracle_score_pairs.restype = ctypes.c_int
+        L.oracle_score_pairs.argtypes = [vp, i64, i64, i64, vp, vp, i64, vp]
         L.oracle_decay.restype = None
         L.oracle_decay.argtypes = [vp, i64, f32]
         L.oracle_order_key.restype = ctypes.c_uint32
@@ -87,6 +89,18 @@ def score(logits: torch.Tensor, ids: torch.Tensor) -> torch.Tensor:
     out = torch.empty(T, dtype=torch.float32)
     stride = logits.stride(0) if T > 1 else V
     lib().oracle_score(logits.data_ptr(), _logits_dtype(logits), T, V, stride, _ptr(ids), _ptr(out))
+    return out
+
+
+def score_pairs(pairs: torch.Tensor, target_logit: torch.Tensor, ids: torch.Tensor, vocab: int) -> torch.Tensor:
+    """fp32 scores from per-tile (max, sum exp) pairs ``[T, n_tiles, 2]`` and the target logits."""
+    assert pairs.dtype == torch.float32 and pairs.dim() == 3 and pairs.shape[2] == 2
+    pairs = pairs.contiguous()
+    T, n_tiles = pairs.shape[:2]
+    target_logit = target_logit.to(torch.float32).contiguous()
+    ids = ids.to(torch.int32).contiguous()
+    out = torch.empty(T, dtype=torch.float32)
+    lib().oracle_score_pairs(_ptr(pairs), T, n_tiles, n_tiles, _ptr(target_logit), _ptr(ids), vocab, _ptr(out))
     return out
 
 

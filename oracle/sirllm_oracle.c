@@ -86,6 +86,48 @@ int oracle_score(const void *logits, int dtype, int64_t T, int64_t V, int64_t ro
     return n_bad;
 }
 
+/*
+ * Token Entropy from split-vocabulary partial results (same definition, Section 3.2): when a
+ * logits row is cut into tiles and tile i is summarised by m_i = max of its logits and
+ * s_i = sum over the tile of exp(z - m_i), then sum_v exp(z_v) = sum_i s_i exp(m_i) and
+ *     e = log(sum_i s_i exp(m_i)) - z[x].
+ * pairs = (m_0, s_0, m_1, s_1, ...) in fp32 as a producer would emit them; a tile with
+ * s_i = 0 (fully masked) contributes nothing.  id rules as in oracle_token_entropy.
+ */
+double oracle_entropy_from_pairs(const float *pairs, int64_t n_tiles, float target_logit, int32_t id,
+                                 int64_t V, int *bad_id)
+{
+    if (id == -1)
+        return 0.0;
+    if (id < 0 || (int64_t)id >= V) {
+        if (bad_id)
+            *bad_id = 1;
+        return 0.0;
+    }
+    double M = -INFINITY;
+    for (int64_t i = 0; i < n_tiles; ++i)
+        if (pairs[2 * i + 1] > 0.0f && (double)pairs[2 * i] > M)
+            M = (double)pairs[2 * i];
+    double S = 0.0;
+    for (int64_t i = 0; i < n_tiles; ++i)
+        if (pairs[2 * i + 1] > 0.0f)
+            S += (double)pairs[2 * i + 1] * exp((double)pairs[2 * i] - M);
+    return (M - (double)target_logit) + log(S);
+}
+
+int oracle_score_pairs(const float *pairs, int64_t T, int64_t n_tiles, int64_t pair_row_stride,
+                       const float *target_logit, const int32_t *ids, int64_t V, float *out_e)
+{
+    int n_bad = 0;
+    for (int64_t t = 0; t < T; ++t) {
+        int bad = 0;
+        out_e[t] = (float)oracle_entropy_from_pairs(pairs + 2 * t * pair_row_stride, n_tiles,
+                                                    target_logit[t], ids[t], V, &bad);
+        n_bad += bad;
+    }
+    return n_bad;
+}
+
 /* Memory decay (Section 3.3, E = E x eta_decay; Algorithm 1 applies it once per
  * round, after the round's scores were appended): one fp32 multiply per entry. */
 void oracle_decay(float *E, int64_t l, float eta)
