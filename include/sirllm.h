@@ -106,6 +106,25 @@ int sirllm_score(const sirllm_config *cfg, const void *logits, const int32_t *to
                  const int32_t *n_new, float *out_entropy, void *ws, void *cuda_stream);
 
 /*
+ * Token Entropy without re-reading the logits (Section 3.2: the same e_i, and its remark
+ * that the score is obtained while the token is generated, at no extra cost).  A producer -
+ * an LM-head GEMM whose epilogue reduces each output tile as it is computed - hands over,
+ * for every logits row, n_tiles pairs and the target logit instead of the row itself:
+ *     pairs[row][i] = (m_i, s_i),  m_i = max of tile i's logits,  s_i = sum_tile exp(z - m_i)
+ *     target_logit[row] = z[row][token_ids[row]]
+ * and  e = log(sum_i s_i * exp(m_i)) - target_logit  (natural log, fp64 combine).  A tile
+ * with s_i = 0 (fully masked) is ignored.  Token ids are only checked (-1 -> 0, out of
+ * range -> 0 and SIRLLM_STATUS_TOKEN_RANGE).  Row and stream layout as in sirllm_score.
+ *   pairs            float[2] x [n_streams*max_new][pair_row_stride], 8-byte aligned
+ *   n_tiles          pairs used per row (>= 1);  pair_row_stride >= n_tiles, in pairs
+ *   target_logit     fp32 [n_streams*max_new]
+ */
+int sirllm_score_pairs(const sirllm_config *cfg, const void *pairs, int32_t n_tiles,
+                       int64_t pair_row_stride, const float *target_logit,
+                       const int32_t *token_ids, const int32_t *n_new, float *out_entropy,
+                       void *ws, void *cuda_stream);
+
+/*
  * sirllm_score for callers that cannot allocate device memory.  (The paper has no
  * counterpart; this is a packaging variant of the same kernel.)
  *
@@ -186,6 +205,14 @@ int sirllm_step(const sirllm_config *cfg, const void *logits, const int32_t *tok
                 const int32_t *n_new, float *scores, int64_t *serial, int32_t *live_len,
                 const float *decay, void *k, void *v, int32_t *keep_idx, int32_t *n_keep,
                 float *new_entropy, void *ws, void *cuda_stream);
+
+/* sirllm_step whose scores come from a producer's per-tile pairs (see sirllm_score_pairs)
+ * instead of the logits; everything else as in sirllm_step (Algorithm 1's loop body). */
+int sirllm_step_pairs(const sirllm_config *cfg, const void *pairs, int32_t n_tiles,
+                      int64_t pair_row_stride, const float *target_logit, const int32_t *token_ids,
+                      const int32_t *n_new, float *scores, int64_t *serial, int32_t *live_len,
+                      const float *decay, void *k, void *v, int32_t *keep_idx, int32_t *n_keep,
+                      float *new_entropy, void *ws, void *cuda_stream);
 
 /* sirllm_step with four caller-created cudaEvent_t handles (host array phase_events[4])
  * recorded on the stream before scoring, before selection, before KV compaction and

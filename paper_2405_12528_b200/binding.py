@@ -22,7 +22,7 @@ STATUS_TOKEN_RANGE, STATUS_OVERFLOW, STATUS_TIMEOUT, STATUS_BAD_KEEP = 1, 2, 4, 
 MAX_CAPACITY = 49152
 
 EXPORTS = ["sirllm_workspace_bytes", "sirllm_workspace_init", "sirllm_score", "sirllm_score_static",
-           "sirllm_decay_select",
+           "sirllm_score_pairs", "sirllm_step_pairs", "sirllm_decay_select",
            "sirllm_compact_kv", "sirllm_step", "sirllm_step_phases", "sirllm_step_host",
            "sirllm_status", "sirllm_strerror",
            "sirllm_last_cuda_error"]
@@ -88,6 +88,10 @@ def lib():
         L.sirllm_score.argtypes = [cfgp, vp, vp, vp, vp, vp, vp]
         L.sirllm_score_static.restype = ctypes.c_int
         L.sirllm_score_static.argtypes = [cfgp, vp, vp, vp, vp, vp, vp]
+        L.sirllm_score_pairs.restype = ctypes.c_int
+        L.sirllm_score_pairs.argtypes = [cfgp, vp, i32, ctypes.c_int64, vp, vp, vp, vp, vp, vp]
+        L.sirllm_step_pairs.restype = ctypes.c_int
+        L.sirllm_step_pairs.argtypes = [cfgp, vp, i32, ctypes.c_int64] + [vp] * 15
         L.sirllm_decay_select.restype = ctypes.c_int
         L.sirllm_decay_select.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, i32, vp, vp]
         L.sirllm_compact_kv.restype = ctypes.c_int
@@ -179,6 +183,44 @@ def sirllm_score_static(cfg: Config, logits, token_ids, n_new, out_entropy, stat
                                      _dev(n_new, torch.int32, "n_new"),
                                      _dev(out_entropy, torch.float32, "out_entropy"),
                                      _dev(status, torch.int32, "status"), _stream()))
+
+
+def _pairs_args(pairs: torch.Tensor):
+    if pairs.dim() != 3 or pairs.shape[2] != 2 or pairs.stride(2) != 1 or pairs.stride(1) != 2:
+        raise SirllmError(ERR_ALIGN, "pairs must be [rows, n_tiles, 2] with contiguous pairs")
+    stride = pairs.stride(0) // 2 if pairs.shape[0] > 1 else pairs.shape[1]
+    if not pairs.is_cuda or pairs.dtype != torch.float32:
+        raise SirllmError(ERR_BAD_CONFIG, "pairs must be a float32 CUDA tensor")
+    return pairs.data_ptr(), int(pairs.shape[1]), int(stride)
+
+
+def sirllm_score_pairs(cfg: Config, pairs, target_logit, token_ids, n_new, out_entropy, ws) -> None:
+    """Scores from per-tile ``(max, sum exp)`` pairs ``[rows, n_tiles, 2]`` and target logits."""
+    ptr, n_tiles, stride = _pairs_args(pairs)
+    _check(lib().sirllm_score_pairs(ctypes.byref(cfg), ptr, n_tiles, stride,
+                                    _dev(target_logit, torch.float32, "target_logit"),
+                                    _dev(token_ids, torch.int32, "token_ids"),
+                                    _dev(n_new, torch.int32, "n_new"),
+                                    _dev(out_entropy, torch.float32, "out_entropy"),
+                                    _dev(ws, torch.uint8, "ws"), _stream()))
+
+
+def sirllm_step_pairs(cfg: Config, pairs, target_logit, token_ids, n_new, scores, serial, live_len,
+                      decay, k, v, keep_idx, n_keep, new_entropy, ws) -> None:
+    ptr, n_tiles, stride = _pairs_args(pairs)
+    _check(lib().sirllm_step_pairs(ctypes.byref(cfg), ptr, n_tiles, stride,
+                                   _dev(target_logit, torch.float32, "target_logit"),
+                                   _dev(token_ids, torch.int32, "token_ids"),
+                                   _dev(n_new, torch.int32, "n_new"),
+                                   _dev(scores, torch.float32, "scores"),
+                                   _dev(serial, torch.int64, "serial"),
+                                   _dev(live_len, torch.int32, "live_len"),
+                                   _dev(decay, torch.float32, "decay"),
+                                   _dev(k, _KV, "k"), _dev(v, _KV, "v"),
+                                   _dev(keep_idx, torch.int32, "keep_idx"),
+                                   _dev(n_keep, torch.int32, "n_keep"),
+                                   _dev(new_entropy, torch.float32, "new_entropy"),
+                                   _dev(ws, torch.uint8, "ws"), _stream()))
 
 
 def sirllm_decay_select(cfg: Config, scores, serial, live_len, decay, keep_idx, n_keep,

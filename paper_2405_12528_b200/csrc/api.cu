@@ -211,21 +211,64 @@ int sirllm_compact_kv(const sirllm_config* cfg, const void* k_src, const void* v
     return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "compact");
 }
 
-static int step_impl(const sirllm_config* cfg, const void* logits, const int32_t* token_ids,
+// Where the round's scores come from: the logits, or a producer's per-tile pairs.
+struct ScoreSource {
+    const void* logits = nullptr;
+    const float2* pairs = nullptr;
+    const float* target_logit = nullptr;
+    int32_t n_tiles = 0;
+    int64_t pair_row_stride = 0;
+};
+
+static int check_pairs(const ScoreSource& src) {
+    if (!src.pairs || !src.target_logit) return SIRLLM_ERR_NULL;
+    if (src.n_tiles < 1 || src.pair_row_stride < src.n_tiles) return SIRLLM_ERR_BAD_CONFIG;
+    if (misaligned(src.pairs, 8) || misaligned(src.target_logit, 4)) return SIRLLM_ERR_ALIGN;
+    return SIRLLM_OK;
+}
+
+static PairScoreParams pair_params(const sirllm_config& c, const ScoreSource& src,
+                                   const int32_t* ids, const int32_t* n_new, void* ws) {
+    PairScoreParams pp;
+    memset(&pp, 0, sizeof pp);
+    pp.pairs = src.pairs;
+    pp.target_logit = src.target_logit;
+    pp.token_ids = ids;
+    pp.n_new = n_new;
+    pp.status = (int32_t*)ws;
+    pp.vocab = c.vocab;
+    pp.pair_row_stride = src.pair_row_stride;
+    pp.n_streams = c.n_streams;
+    pp.max_new = c.max_new;
+    pp.n_tiles = src.n_tiles;
+    pp.capacity = c.capacity;
+    return pp;
+}
+
+static int step_impl(const sirllm_config* cfg, const ScoreSource& src, const int32_t* token_ids,
                      const int32_t* n_new, float* scores, int64_t* serial, int32_t* live_len,
                      const float* decay, void* k, void* v, int32_t* keep_idx, int32_t* n_keep,
                      float* new_entropy, void* ws, void* cuda_stream, void** ev) {
     int rc = validate_config(cfg);
     if (rc != SIRLLM_OK) return rc;
-    if (!logits || !token_ids || !scores || !live_len || !decay || !ws) return SIRLLM_ERR_NULL;
+    if (!token_ids || !scores || !live_len || !decay || !ws) return SIRLLM_ERR_NULL;
     if (misaligned(ws, 256)) return SIRLLM_ERR_ALIGN;
-    if ((rc = check_logits(*cfg, logits)) != SIRLLM_OK) return rc;
+    if (src.pairs == nullptr) {
+        if (!src.logits) return SIRLLM_ERR_NULL;
+        if ((rc = check_logits(*cfg, src.logits)) != SIRLLM_OK) return rc;
+    } else if ((rc = check_pairs(src)) != SIRLLM_OK) {
+        return rc;
+    }
     const WorkspaceLayout L = workspace_layout(*cfg);
     SelectParams sp = select_params(*cfg, L, scores, serial, live_len, decay, keep_idx, n_keep, ws);
-    ScoreParams sc = score_params(*cfg, L, logits, token_ids, n_new, ws);
+    ScoreParams sc = score_params(*cfg, L, src.logits, token_ids, n_new, ws);
     sc.out_entropy = new_entropy;
     sc.scores = scores;
     sc.live_len = live_len;
+    PairScoreParams pp = pair_params(*cfg, src, token_ids, n_new, ws);
+    pp.out_entropy = new_entropy;
+    pp.scores = scores;
+    pp.live_len = live_len;
     sp.n_new = n_new;
     sp.max_new = cfg->max_new;
     sp.compact_scores = 1;
@@ -239,7 +282,7 @@ static int step_impl(const sirllm_config* cfg, const void* logits, const int32_t
     if (ev && (e = cudaEventRecord((cudaEvent_t)ev[i], st)) != cudaSuccess) \
         return cuda_fail(e, "cudaEventRecord");
     SIRLLM_MARK(0)
-    e = launch_score(sc, st);
+    e = src.pairs ? launch_score_pairs(pp, st) : launch_score(sc, st);
     if (e != cudaSuccess) return cuda_fail(e, "score");
     SIRLLM_MARK(1)
     e = launch_select(sp, cfg->n_streams, st, ev == nullptr);
@@ -256,7 +299,44 @@ int sirllm_step(const sirllm_config* cfg, const void* logits, const int32_t* tok
                 const int32_t* n_new, float* scores, int64_t* serial, int32_t* live_len,
                 const float* decay, void* k, void* v, int32_t* keep_idx, int32_t* n_keep,
                 float* new_entropy, void* ws, void* cuda_stream) {
-    return step_impl(cfg, logits, token_ids, n_new, scores, serial, live_len, decay, k, v, keep_idx,
+    ScoreSource src;
+    src.logits = logits;
+    return step_impl(cfg, src, token_ids, n_new, scores, serial, live_len, decay, k, v, keep_idx,
+                     n_keep, new_entropy, ws, cuda_stream, nullptr);
+}
+
+int sirllm_score_pairs(const sirllm_config* cfg, const void* pairs, int32_t n_tiles,
+                       int64_t pair_row_stride, const float* target_logit,
+                       const int32_t* token_ids, const int32_t* n_new, float* out_entropy,
+                       void* ws, void* cuda_stream) {
+    int rc = validate_config(cfg);
+    if (rc != SIRLLM_OK) return rc;
+    if (!token_ids || !out_entropy || !ws) return SIRLLM_ERR_NULL;
+    if (misaligned(ws, 256)) return SIRLLM_ERR_ALIGN;
+    ScoreSource src;
+    src.pairs = (const float2*)pairs;
+    src.target_logit = target_logit;
+    src.n_tiles = n_tiles;
+    src.pair_row_stride = pair_row_stride;
+    if ((rc = check_pairs(src)) != SIRLLM_OK) return rc;
+    PairScoreParams pp = pair_params(*cfg, src, token_ids, n_new, ws);
+    pp.out_entropy = out_entropy;
+    cudaError_t e = launch_score_pairs(pp, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "score_pairs");
+}
+
+int sirllm_step_pairs(const sirllm_config* cfg, const void* pairs, int32_t n_tiles,
+                      int64_t pair_row_stride, const float* target_logit, const int32_t* token_ids,
+                      const int32_t* n_new, float* scores, int64_t* serial, int32_t* live_len,
+                      const float* decay, void* k, void* v, int32_t* keep_idx, int32_t* n_keep,
+                      float* new_entropy, void* ws, void* cuda_stream) {
+    ScoreSource src;
+    src.pairs = (const float2*)pairs;
+    src.target_logit = target_logit;
+    src.n_tiles = n_tiles;
+    src.pair_row_stride = pair_row_stride;
+    if (!pairs) return SIRLLM_ERR_NULL;
+    return step_impl(cfg, src, token_ids, n_new, scores, serial, live_len, decay, k, v, keep_idx,
                      n_keep, new_entropy, ws, cuda_stream, nullptr);
 }
 
@@ -267,7 +347,9 @@ int sirllm_step_phases(const sirllm_config* cfg, const void* logits, const int32
     if (!phase_events) return SIRLLM_ERR_NULL;
     for (int i = 0; i < 4; ++i)
         if (!phase_events[i]) return SIRLLM_ERR_NULL;
-    return step_impl(cfg, logits, token_ids, n_new, scores, serial, live_len, decay, k, v, keep_idx,
+    ScoreSource src;
+    src.logits = logits;
+    return step_impl(cfg, src, token_ids, n_new, scores, serial, live_len, decay, k, v, keep_idx,
                      n_keep, new_entropy, ws, cuda_stream, phase_events);
 }
 
@@ -325,7 +407,9 @@ int sirllm_step_host(const sirllm_config* cfg, const void* h_logits, const int32
     if (e != cudaSuccess) return cuda_fail(e, "ids H2D");
     e = cudaMemcpyAsync(d_n_new, h_n_new, (size_t)cfg->n_streams * 4, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(e, "n_new H2D");
-    rc = step_impl(cfg, d_logits, d_token_ids, d_n_new, scores, serial, live_len, decay, k, v,
+    ScoreSource src;
+    src.logits = d_logits;
+    rc = step_impl(cfg, src, d_token_ids, d_n_new, scores, serial, live_len, decay, k, v,
                    keep_idx, n_keep, new_entropy, ws, cuda_stream, nullptr);
     if (rc != SIRLLM_OK) return rc;
     e = cudaMemcpyAsync(h_keep_idx, keep_idx, (size_t)cfg->n_streams * cfg->threshold * 4,

@@ -54,6 +54,19 @@ struct ScoreParams {
     int32_t n_streams, max_new, n_part, logits_dtype, capacity;
 };
 
+struct PairScoreParams {
+    const float2* pairs;        // [rows][pair_row_stride] (tile max, tile sum of exp(z - max))
+    const float* target_logit;  // [rows]
+    const int32_t* token_ids;
+    const int32_t* n_new;       // nullable
+    int32_t* status;
+    float* out_entropy;         // nullable
+    float* scores;              // nullable: append at scores[s][live_len[s] + t]
+    const int32_t* live_len;
+    int64_t vocab, pair_row_stride;
+    int32_t n_streams, max_new, n_tiles, capacity;
+};
+
 struct SelectParams {
     const int32_t* n_new;  // with score_new: tokens appended this round (nullable: max_new)
     int32_t max_new;
@@ -87,6 +100,7 @@ struct CompactParams {
 };
 
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st);
+cudaError_t launch_score_pairs(const PairScoreParams& p, cudaStream_t st);
 // `overlap`: launch with programmatic stream serialization, so the grid may become resident
 // while the previous kernel on the stream drains; the kernel itself waits for that kernel's
 // results (grid_dependency_wait) before it reads them.

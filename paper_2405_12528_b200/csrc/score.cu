@@ -213,7 +213,59 @@ score_kernel(const ScoreParams p) {
     }
 }
 
+// Token Entropy from split-vocabulary partial results: a producer (an LM-head GEMM whose
+// epilogue reduces every output tile) hands over, per row, n_tiles pairs
+// (m_i = tile max, s_i = sum exp(z - m_i)) and the target logit, so the logits row itself is
+// never read.  One warp per row; fp64 combine in a fixed order.
+__global__ void __launch_bounds__(128) score_pairs_kernel(const PairScoreParams p) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    grid_launch_dependents();
+    if (row >= (int64_t)p.n_streams * p.max_new) return;
+    const int s = (int)(row / p.max_new);
+    const int t = (int)(row - (int64_t)s * p.max_new);
+    int T = p.max_new;
+    if (p.n_new != nullptr) T = min(p.n_new[s], p.max_new);
+    if (t >= T) return;
+    const float2* pr = p.pairs + row * p.pair_row_stride;
+    float M = kNegHuge;
+    for (int i = lane; i < p.n_tiles; i += 32) {
+        const float2 q = pr[i];
+        if (q.y > 0.f) M = fmaxf(M, q.x);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, o));
+    double acc = 0.0;
+    for (int i = lane; i < p.n_tiles; i += 32) {
+        const float2 q = pr[i];
+        if (q.y > 0.f) acc += (double)q.y * exp((double)q.x - (double)M);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    if (lane == 0) {
+        const int32_t id = p.token_ids[row];
+        float e = 0.f;
+        if (id >= 0 && (int64_t)id < p.vocab) {
+            e = fmaxf((float)(((double)M - (double)p.target_logit[row]) + log(acc)), 0.0f);
+        } else if (id != -1) {
+            atomicOr(p.status, SIRLLM_STATUS_TOKEN_RANGE);
+        }
+        if (p.out_entropy) p.out_entropy[row] = e;
+        if (p.scores != nullptr) {
+            const int l0 = p.live_len[s];
+            if (l0 >= 0 && l0 <= p.capacity - T) p.scores[(size_t)s * p.capacity + l0 + t] = e;
+        }
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_score_pairs(const PairScoreParams& p, cudaStream_t st) {
+    const int64_t rows = (int64_t)p.n_streams * p.max_new;
+    if (rows == 0) return cudaSuccess;
+    score_pairs_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(p);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
     const int64_t ctas = (int64_t)p.n_streams * p.max_new * p.n_part;

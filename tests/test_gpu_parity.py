@@ -322,3 +322,73 @@ def test_step_overflowing_round_is_skipped_and_flagged():
     assert B.sirllm_status(st.ws, clear=True) == B.STATUS_OVERFLOW
     assert st.host_len == [200, 250]
     assert torch.equal(st.scores[0], snap[0][0]) and torch.equal(st.k[0], snap[1][0])
+
+
+# ------------------------------------------------------------------------------- scores from pairs
+
+def _device_tile_pairs(logits, tile):
+    """What a GEMM epilogue would emit: per-tile (max, sum exp(z - max)) in fp32 (torch ops,
+    input preparation only)."""
+    T, V = logits.shape
+    n = (V + tile - 1) // tile
+    z = torch.full((T, n * tile), float("-inf"), dtype=torch.float32, device=logits.device)
+    z[:, :V] = logits.float()
+    z = z.view(T, n, tile)
+    m = z.max(dim=2).values
+    s = torch.exp(z - m[:, :, None]).sum(dim=2)
+    return torch.stack([m, s], dim=2).contiguous()
+
+
+@pytest.mark.parametrize("tile", [128, 1000])
+def test_score_pairs_matches_oracle_and_the_logits_path(tile):
+    S, M, V = 2, 50, 32000
+    cfg = _score_cfg(M, V, torch.bfloat16, n_streams=S)
+    ws = B.new_workspace(cfg)
+    g = torch.Generator().manual_seed(tile)
+    logits = (torch.randn(S * M, V, generator=g) * 2.5).to(torch.bfloat16).to(DEV)
+    ids = torch.randint(0, V, (S * M,), generator=g, dtype=torch.int32)
+    ids[3], ids[60] = -1, V
+    d_ids = ids.to(DEV)
+    n_new = torch.tensor([50, 17], dtype=torch.int32, device=DEV)
+    pairs = _device_tile_pairs(logits, tile)
+    target = logits.float()[torch.arange(S * M, device=DEV), d_ids.long().clamp(0, V - 1)].contiguous()
+    out = torch.full((S * M,), -2.0, device=DEV)
+    B.sirllm_score_pairs(cfg, pairs, target, d_ids, n_new, out, ws)
+    assert B.sirllm_status(ws, clear=True) == 0          # row 60 is beyond n_new[1]: not looked at
+    live = torch.zeros(S * M, dtype=torch.bool)
+    live[:50] = True
+    live[50:67] = True
+    want = oracle.score_pairs(pairs.cpu(), target.cpu(), ids, V)
+    assert_entropy_close(out.cpu()[live], want[live])
+    assert (out.cpu()[~live] == -2.0).all() and float(out[3]) == 0.0
+    ref = torch.zeros(S * M, device=DEV)
+    B.sirllm_score(cfg, logits, d_ids, n_new, ref, ws)
+    assert_entropy_close(out.cpu()[live], ref.cpu()[live])
+
+
+def test_step_pairs_round_matches_oracle_and_the_logits_round():
+    w = wl.WORKLOADS["mistral_7b_gqa"].scaled(n_layers=1, n_kv_heads=2, capacity=1024, budget=512,
+                                              n_recent=64, new_tokens=300, vocab=8000)
+    a, b = DeviceState(w), DeviceState(w)
+    tw = oracle_twin(w, b.decay.cpu(), with_kv=False)[0]
+    for r in range(4):
+        a.fill_round(r)
+        b.fill_round(r)
+        a.step()
+        pairs = _device_tile_pairs(b.logits, 256)
+        target = b.logits.float()[torch.arange(b.logits.shape[0], device=DEV),
+                                  b.token_ids.long()].contiguous()
+        B.sirllm_step_pairs(b.cfg, pairs, target, b.token_ids, b.n_new, b.scores, b.serial, b.live_len,
+                            b.decay, b.k, b.v, b.keep_idx, b.n_keep, b.new_entropy, b.ws)
+        b.host_len = b.live_len.cpu().tolist()
+        assert B.sirllm_status(b.ws) == 0
+        e = b.new_entropy[:300].cpu()
+        assert_entropy_close(e, oracle.score_pairs(pairs.cpu(), target.cpu(), b.token_ids.cpu(), w.vocab))
+        assert_entropy_close(e, a.new_entropy[:300])            # the logits path agrees
+        keep = tw.step(e)                                       # the oracle ranks the same scores
+        n = tw.live_len
+        assert b.host_len == [n] and a.host_len == [n]
+        assert torch.equal(b.keep_idx[0, :n].cpu(), keep)
+        assert torch.equal(b.scores[0, :n].cpu().view(torch.int32), tw.E[:n].view(torch.int32))
+        assert torch.equal(b.serial[0, :n].cpu(), tw.serial[:n])
+        b.check_kv_by_content()
