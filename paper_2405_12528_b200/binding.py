@@ -91,7 +91,7 @@ def lib():
         L.sirllm_score_pairs.restype = ctypes.c_int
         L.sirllm_score_pairs.argtypes = [cfgp, vp, i32, ctypes.c_int64, vp, vp, vp, vp, vp, vp]
         L.sirllm_step_pairs.restype = ctypes.c_int
-        L.sirllm_step_pairs.argtypes = [cfgp, vp, i32, ctypes.c_int64] + [vp] * 15
+        L.sirllm_step_pairs.argtypes = [cfgp, vp, i32, ctypes.c_int64] + [vp] * 14
         L.sirllm_decay_select.restype = ctypes.c_int
         L.sirllm_decay_select.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, i32, vp, vp]
         L.sirllm_compact_kv.restype = ctypes.c_int

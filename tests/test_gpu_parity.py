@@ -347,20 +347,20 @@ def test_score_pairs_matches_oracle_and_the_logits_path(tile):
     g = torch.Generator().manual_seed(tile)
     logits = (torch.randn(S * M, V, generator=g) * 2.5).to(torch.bfloat16).to(DEV)
     ids = torch.randint(0, V, (S * M,), generator=g, dtype=torch.int32)
-    ids[3], ids[60] = -1, V
+    ids[3], ids[60], ids[75] = -1, V, V          # row 75 lies beyond n_new[1]: never looked at
     d_ids = ids.to(DEV)
     n_new = torch.tensor([50, 17], dtype=torch.int32, device=DEV)
     pairs = _device_tile_pairs(logits, tile)
     target = logits.float()[torch.arange(S * M, device=DEV), d_ids.long().clamp(0, V - 1)].contiguous()
     out = torch.full((S * M,), -2.0, device=DEV)
     B.sirllm_score_pairs(cfg, pairs, target, d_ids, n_new, out, ws)
-    assert B.sirllm_status(ws, clear=True) == 0          # row 60 is beyond n_new[1]: not looked at
+    assert B.sirllm_status(ws, clear=True) == B.STATUS_TOKEN_RANGE      # from row 60
     live = torch.zeros(S * M, dtype=torch.bool)
     live[:50] = True
     live[50:67] = True
     want = oracle.score_pairs(pairs.cpu(), target.cpu(), ids, V)
     assert_entropy_close(out.cpu()[live], want[live])
-    assert (out.cpu()[~live] == -2.0).all() and float(out[3]) == 0.0
+    assert (out.cpu()[~live] == -2.0).all() and float(out[3]) == 0.0 and float(out[60]) == 0.0
     ref = torch.zeros(S * M, device=DEV)
     B.sirllm_score(cfg, logits, d_ids, n_new, ref, ws)
     assert_entropy_close(out.cpu()[live], ref.cpu()[live])
