@@ -53,6 +53,14 @@ def lib():
         L.oracle_step.restype = i32
         L.oracle_step.argtypes = [vp, i32, vp, vp, vp, i32, f32, i32, i32, i32, i32, i32, vp, vp,
                                   i64, i64, vp]
+        L.oracle_keep_stream.restype = i32
+        L.oracle_keep_stream.argtypes = [i32, i32, i32, i32, vp]
+        L.oracle_keep_interval.restype = i32
+        L.oracle_keep_interval.argtypes = [i32, i32, i32, i32, i32, vp]
+        L.oracle_philox4x32_10.restype = None
+        L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
+        L.oracle_keep_random.restype = i32
+        L.oracle_keep_random.argtypes = [i32, i32, i32, i32, i32, ctypes.c_uint64, i32, i32, vp]
         _lib = L
     return _lib
 
@@ -134,6 +142,34 @@ def gather_rows(src: torch.Tensor, keep: torch.Tensor) -> torch.Tensor:
     row_bytes = src[0].numel() * src.element_size() if src.shape[0] else 0
     lib().oracle_gather_rows(_ptr(src), _ptr(out), row_bytes, _ptr(keep), keep.numel())
     return out
+
+
+STREAM, RANDOM, INTERVAL = 1, 2, 3
+
+
+def philox4x32_10(ctr, key):
+    c = (ctypes.c_uint32 * 4)(*ctr)
+    k = (ctypes.c_uint32 * 2)(*key)
+    out = (ctypes.c_uint32 * 4)()
+    lib().oracle_philox4x32_10(c, k, out)
+    return list(out)
+
+
+def keep_policy(policy: int, live_len: int, n_sink: int, n_recent: int, budget: int,
+                threshold: int | None = None, seed: int = 0, stream: int = 0, rnd: int = 0) -> torch.Tensor:
+    """Keep list (ascending int32) of one of the paper's comparison policies (Section 4.1.1)."""
+    threshold = budget if threshold is None else threshold
+    keep = torch.empty(max(int(live_len), budget, 1), dtype=torch.int32)
+    if policy == STREAM:
+        n = lib().oracle_keep_stream(live_len, n_sink, budget, threshold, _ptr(keep))
+    elif policy == INTERVAL:
+        n = lib().oracle_keep_interval(live_len, n_sink, n_recent, budget, threshold, _ptr(keep))
+    elif policy == RANDOM:
+        n = lib().oracle_keep_random(live_len, n_sink, n_recent, budget, threshold, seed, stream, rnd,
+                                     _ptr(keep))
+    else:
+        raise ValueError("unknown policy")
+    return keep[:n].clone()
 
 
 class Stream:

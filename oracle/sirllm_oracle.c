@@ -274,3 +274,97 @@ int32_t oracle_step(const float *new_e, int32_t T, float *E, int64_t *serial, in
     free(tmp);
     return n_keep;
 }
+
+/* ---- the paper's comparison policies (Section 4.1.1) as keep-list generators ---------
+ * They feed the same K/V gather as the entropy selection.  All use the trigger of
+ * Algorithm 1 (nothing is evicted while l <= threshold) and list the kept slots ascending. */
+
+/* StreamLLM (Sections 3.1, 4.1.1): the sink tokens and the most recent tokens only,
+ * budget slots in all. */
+int32_t oracle_keep_stream(int32_t l, int32_t n_sink, int32_t budget, int32_t threshold, int32_t *keep)
+{
+    if (l <= threshold) {
+        for (int32_t i = 0; i < l; ++i)
+            keep[i] = i;
+        return l;
+    }
+    int32_t n = 0;
+    for (int32_t i = 0; i < n_sink; ++i)
+        keep[n++] = i;
+    for (int32_t i = l - (budget - n_sink); i < l; ++i)
+        keep[n++] = i;
+    return n;
+}
+
+/* IntervalLLM (Section 4.1.1): the sink tokens, then one historical token every `interval`
+ * slots, interval = floor(history length / cache size), until the cache is full.  The
+ * configured recent window (0 in the paper's rows) is kept as in the entropy policy. */
+int32_t oracle_keep_interval(int32_t l, int32_t n_sink, int32_t n_recent, int32_t budget,
+                             int32_t threshold, int32_t *keep)
+{
+    if (l <= threshold) {
+        for (int32_t i = 0; i < l; ++i)
+            keep[i] = i;
+        return l;
+    }
+    int32_t interval = l / budget;
+    int32_t k = budget - n_sink - n_recent, n = 0;
+    for (int32_t i = 0; i < n_sink; ++i)
+        keep[n++] = i;
+    for (int32_t i = n_sink, taken = 0; i < l - n_recent && taken < k; i += interval, ++taken)
+        keep[n++] = i;
+    for (int32_t i = l - n_recent; i < l; ++i)
+        keep[n++] = i;
+    return n;
+}
+
+/* Philox4x32-10 counter-based generator (Salmon, Moraes, Dror, Shaw, "Parallel random
+ * numbers: as easy as 1, 2, 3", SC'11): ten rounds of two 32x32->64 multiplies. */
+void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int r = 0; r < 10; ++r) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1, n3 = (uint32_t)p0;
+        c0 = n0, c1 = n1, c2 = n2, c3 = n3;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0, out[1] = c1, out[2] = c2, out[3] = c3;
+}
+
+/* RandomLLM (Section 4.1.1): the sink tokens and a uniformly random choice of k historical
+ * tokens.  Slot i of the middle draws the 24-bit number
+ *     u_i = philox(counter = (i, round, stream, 0), key = seed)[0] >> 8
+ * and the k largest stay (equal draws: the lower slot), which is a uniform k-subset. */
+int32_t oracle_keep_random(int32_t l, int32_t n_sink, int32_t n_recent, int32_t budget,
+                           int32_t threshold, uint64_t seed, int32_t stream, int32_t round,
+                           int32_t *keep)
+{
+    if (l <= threshold) {
+        for (int32_t i = 0; i < l; ++i)
+            keep[i] = i;
+        return l;
+    }
+    int32_t lo = n_sink, hi = l - n_recent, k = budget - n_sink - n_recent, n_mid = hi - lo;
+    ranked_t *mid = malloc(sizeof(ranked_t) * (size_t)(n_mid > 0 ? n_mid : 1));
+    uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    for (int32_t i = lo; i < hi; ++i) {
+        uint32_t ctr[4] = {(uint32_t)i, (uint32_t)round, (uint32_t)stream, 0u}, out[4];
+        oracle_philox4x32_10(ctr, key, out);
+        mid[i - lo].key = out[0] >> 8;
+        mid[i - lo].slot = i;
+    }
+    qsort(mid, (size_t)n_mid, sizeof(ranked_t), by_score_desc_then_slot_asc);
+    int32_t n = 0;
+    for (int32_t i = 0; i < lo; ++i)
+        keep[n++] = i;
+    for (int32_t r = 0; r < k; ++r)
+        keep[n++] = mid[r].slot;
+    for (int32_t i = hi; i < l; ++i)
+        keep[n++] = i;
+    free(mid);
+    qsort(keep, (size_t)n, sizeof(int32_t), by_int_asc);
+    return n;
+}
