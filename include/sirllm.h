@@ -57,6 +57,11 @@ extern "C" {
 #define SIRLLM_STATUS_BAD_KEEP 8    /* a caller-supplied keep list is not strictly ascending within
                                        [0, capacity); that stream was not compacted */
 
+/* comparison policies of Section 4.1.1 for sirllm_keep_policy */
+#define SIRLLM_POLICY_STREAM 1
+#define SIRLLM_POLICY_RANDOM 2
+#define SIRLLM_POLICY_INTERVAL 3
+
 /* Largest `capacity` the selection kernel supports (the scores of one stream are
  * held in one SM's shared memory). */
 #define SIRLLM_MAX_CAPACITY 49152
@@ -176,6 +181,25 @@ int sirllm_score_static(const sirllm_config *cfg, const void *logits, const int3
 int sirllm_decay_select(const sirllm_config *cfg, float *scores, int64_t *serial, int32_t *live_len,
                         const float *decay, int32_t *keep_idx, int32_t *n_keep,
                         int32_t compact_scores, void *ws, void *cuda_stream);
+
+/*
+ * Keep lists of the paper's comparison policies (Section 4.1.1), in the format of
+ * sirllm_decay_select so that they feed sirllm_compact_kv unchanged.  Nothing is evicted
+ * while live_len[s] <= threshold (identity list); otherwise, in ascending order,
+ *   SIRLLM_POLICY_STREAM    sinks and the most recent budget - n_sink slots (StreamLLM)
+ *   SIRLLM_POLICY_INTERVAL  sinks, then every interval-th slot behind them, interval =
+ *                           floor(live_len / budget), until k = budget - n_sink - n_recent
+ *                           are taken, then the recent window (IntervalLLM)
+ *   SIRLLM_POLICY_RANDOM    sinks, a uniformly random k-subset of the middle, the recent
+ *                           window (RandomLLM).  Middle slot i draws the 24-bit number
+ *                           philox4x32_10(counter = (i, round, stream_base + s, 0),
+ *                           key = seed)[0] >> 8; the k largest stay, equal draws -> lower slot.
+ * Scores, tags and live_len are not touched: these policies do not use them; the caller
+ * sets live_len[s] = n_keep[s] after compacting.
+ */
+int sirllm_keep_policy(const sirllm_config *cfg, int32_t policy, const int32_t *live_len,
+                       uint64_t seed, int32_t round, int32_t stream_base, int32_t *keep_idx,
+                       int32_t *n_keep, void *ws, void *cuda_stream);
 
 /*
  * KV gather (Section 3.1, X[Id]; Section 3.3, KV_cache = KV_cache[Id_sink, Id_entropy]):

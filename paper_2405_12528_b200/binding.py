@@ -20,9 +20,10 @@ F32, BF16, F16 = 0, 1, 2
 OK, ERR_NULL, ERR_BAD_CONFIG, ERR_ALIGN, ERR_CUDA, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5
 STATUS_TOKEN_RANGE, STATUS_OVERFLOW, STATUS_TIMEOUT, STATUS_BAD_KEEP = 1, 2, 4, 8
 MAX_CAPACITY = 49152
+POLICY_STREAM, POLICY_RANDOM, POLICY_INTERVAL = 1, 2, 3
 
 EXPORTS = ["sirllm_workspace_bytes", "sirllm_workspace_init", "sirllm_score", "sirllm_score_static",
-           "sirllm_score_pairs", "sirllm_step_pairs", "sirllm_decay_select",
+           "sirllm_score_pairs", "sirllm_step_pairs", "sirllm_decay_select", "sirllm_keep_policy",
            "sirllm_compact_kv", "sirllm_step", "sirllm_step_phases", "sirllm_step_host",
            "sirllm_status", "sirllm_strerror",
            "sirllm_last_cuda_error"]
@@ -94,6 +95,8 @@ def lib():
         L.sirllm_step_pairs.argtypes = [cfgp, vp, i32, ctypes.c_int64] + [vp] * 14
         L.sirllm_decay_select.restype = ctypes.c_int
         L.sirllm_decay_select.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, i32, vp, vp]
+        L.sirllm_keep_policy.restype = ctypes.c_int
+        L.sirllm_keep_policy.argtypes = [cfgp, i32, vp, ctypes.c_uint64, i32, i32, vp, vp, vp, vp]
         L.sirllm_compact_kv.restype = ctypes.c_int
         L.sirllm_compact_kv.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.sirllm_step.restype = ctypes.c_int
@@ -232,6 +235,16 @@ def sirllm_decay_select(cfg: Config, scores, serial, live_len, decay, keep_idx, 
                                      _dev(keep_idx, torch.int32, "keep_idx"),
                                      _dev(n_keep, torch.int32, "n_keep"),
                                      int(bool(compact_scores)), _dev(ws, torch.uint8, "ws"), _stream()))
+
+
+def sirllm_keep_policy(cfg: Config, policy: int, live_len, seed: int, rnd: int, stream_base: int,
+                       keep_idx, n_keep, ws) -> None:
+    """Keep lists of StreamLLM / RandomLLM / IntervalLLM (``POLICY_*``) for ``sirllm_compact_kv``."""
+    _check(lib().sirllm_keep_policy(ctypes.byref(cfg), int(policy), _dev(live_len, torch.int32, "live_len"),
+                                    int(seed), int(rnd), int(stream_base),
+                                    _dev(keep_idx, torch.int32, "keep_idx"),
+                                    _dev(n_keep, torch.int32, "n_keep"),
+                                    _dev(ws, torch.uint8, "ws"), _stream()))
 
 
 _KV = (torch.bfloat16, torch.float16)

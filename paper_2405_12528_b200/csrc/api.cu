@@ -54,6 +54,10 @@ WorkspaceLayout workspace_layout(const sirllm_config& c) {
     off = align_up(off + (size_t)c.n_streams * c.threshold * 4, 256);
     L.tickets_off = off;
     off = align_up(off + (size_t)c.n_streams * c.max_new * 4, 256);
+    L.policy_ranks_off = off;
+    off = align_up(off + (size_t)c.n_streams * c.capacity * 4, 256);
+    L.policy_ones_off = off;
+    off = align_up(off + (size_t)c.n_streams * 4, 256);
     L.partials_off = off;
     off = align_up(off + (size_t)c.n_streams * c.max_new * L.n_part * sizeof(float2), 256);
     L.total = off;
@@ -157,6 +161,39 @@ int sirllm_decay_select(const sirllm_config* cfg, float* scores, int64_t* serial
     p.compact_scores = compact_scores != 0;
     p.score_new = 0;
     cudaError_t e = launch_select(p, cfg->n_streams, (cudaStream_t)cuda_stream, false);
+    return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "select");
+}
+
+static int keep_policy_impl(const sirllm_config* cfg, int32_t policy, const int32_t* live_len,
+                            uint64_t seed, int32_t round, int32_t stream_base, int32_t* keep_idx,
+                            int32_t* n_keep, void* ws, void* cuda_stream) {
+    int rc = validate_config(cfg);
+    if (rc != SIRLLM_OK) return rc;
+    if (!live_len || !keep_idx || !n_keep || !ws) return SIRLLM_ERR_NULL;
+    if (misaligned(ws, 256)) return SIRLLM_ERR_ALIGN;
+    if (policy != SIRLLM_POLICY_STREAM && policy != SIRLLM_POLICY_RANDOM &&
+        policy != SIRLLM_POLICY_INTERVAL)
+        return SIRLLM_ERR_BAD_CONFIG;
+    const WorkspaceLayout L = workspace_layout(*cfg);
+    PolicyParams pp;
+    pp.live_len = live_len;
+    pp.ranks = (float*)((char*)ws + L.policy_ranks_off);
+    pp.ones = (float*)((char*)ws + L.policy_ones_off);
+    pp.seed = seed;
+    pp.policy = policy;
+    pp.round = round;
+    pp.stream_base = stream_base;
+    pp.capacity = cfg->capacity;
+    pp.budget = cfg->budget;
+    pp.n_sink = cfg->n_sink;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = launch_policy_ranks(pp, cfg->n_streams, st);
+    if (e != cudaSuccess) return cuda_fail(e, "policy_ranks");
+    SelectParams sp = select_params(*cfg, L, pp.ranks, nullptr, const_cast<int32_t*>(live_len),
+                                    pp.ones, keep_idx, n_keep, ws);
+    sp.compact_scores = 0;  // live_len is only read
+    sp.score_new = 0;
+    e = launch_select(sp, cfg->n_streams, st, false);
     return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "select");
 }
 
@@ -420,6 +457,13 @@ int sirllm_step_host(const sirllm_config* cfg, const void* h_logits, const int32
     e = cudaMemcpyAsync(h_new_entropy, new_entropy, n_rows * 4, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return cuda_fail(e, "entropy D2H");
     return SIRLLM_OK;
+}
+
+int sirllm_keep_policy(const sirllm_config* cfg, int32_t policy, const int32_t* live_len,
+                       uint64_t seed, int32_t round, int32_t stream_base, int32_t* keep_idx,
+                       int32_t* n_keep, void* ws, void* cuda_stream) {
+    return keep_policy_impl(cfg, policy, live_len, seed, round, stream_base, keep_idx, n_keep,
+                                   ws, cuda_stream);
 }
 
 int sirllm_status(void* ws, void* cuda_stream, int32_t* status_out, int32_t clear) {

@@ -14,6 +14,7 @@ namespace sirllm {
 //   first_moved[n_streams]                first slot whose row changes place when compacting
 //   n_keep_fallback[n_streams]            used when the caller passes no n_keep
 //   keep_fallback[n_streams][threshold]   used when the caller passes no keep_idx
+//   policy_ranks[n_streams][capacity]     synthetic scores of the comparison policies, ones[n_streams]
 //   tickets[n_streams*max_new]            arrivals per logits row (the last CTA finishes the row)
 //   partials[n_streams*max_new][n_part]   (scaled max, sum) pair per CTA of a multi-CTA row
 struct WorkspaceLayout {
@@ -22,6 +23,8 @@ struct WorkspaceLayout {
     size_t n_keep_off;
     size_t keep_off;
     size_t tickets_off;
+    size_t policy_ranks_off;
+    size_t policy_ones_off;
     size_t partials_off;
     size_t total;
     int32_t n_part;  // CTAs (groups of kScoreWarpsPerCta segments) per logits row
@@ -84,6 +87,14 @@ struct SelectParams {
     int32_t score_new;       // the round's new scores were appended behind live_len by the scorer
 };
 
+struct PolicyParams {
+    const int32_t* live_len;
+    float* ranks;  // [n_streams][capacity] synthetic scores
+    float* ones;   // [n_streams] decay ratio 1 for the selection kernel
+    uint64_t seed;
+    int32_t policy, round, stream_base, capacity, budget, n_sink;
+};
+
 struct CompactParams {
     const char* src[2];  // K, V (nullable)
     char* dst[2];
@@ -105,6 +116,7 @@ cudaError_t launch_score_pairs(const PairScoreParams& p, cudaStream_t st);
 // while the previous kernel on the stream drains; the kernel itself waits for that kernel's
 // results (grid_dependency_wait) before it reads them.
 cudaError_t launch_select(const SelectParams& p, int n_streams, cudaStream_t st, bool overlap);
+cudaError_t launch_policy_ranks(const PolicyParams& p, int n_streams, cudaStream_t st);
 cudaError_t launch_compact_plan(const CompactParams& p, int n_streams, int32_t* first_moved,
                                 cudaStream_t st);
 cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap);

@@ -392,3 +392,34 @@ def test_step_pairs_round_matches_oracle_and_the_logits_round():
         assert torch.equal(b.scores[0, :n].cpu().view(torch.int32), tw.E[:n].view(torch.int32))
         assert torch.equal(b.serial[0, :n].cpu(), tw.serial[:n])
         b.check_kv_by_content()
+
+
+# ------------------------------------------------------------------------------- comparison policies
+
+@pytest.mark.parametrize("policy", [B.POLICY_STREAM, B.POLICY_RANDOM, B.POLICY_INTERVAL])
+def test_keep_policy_matches_oracle_and_feeds_the_gather(policy):
+    # StreamLLM / RandomLLM / IntervalLLM of Section 4.1.1: keep lists bit exact, then the same
+    # K/V gather; streams with different lengths, one under the threshold
+    lens = [1078, 1025, 3000, 640, 0]
+    S, cap, budget, n_sink, n_recent = len(lens), 3072, 1024, 4, 0
+    for n_recent in (0, 37):
+        cfg = B.make_config(S, 2, 1, 64, cap, budget, n_sink, n_recent, 0, 16, torch.float32, torch.bfloat16)
+        ws = B.new_workspace(cfg)
+        live = torch.tensor(lens, dtype=torch.int32, device=DEV)
+        keep = torch.full((S, budget), -1, dtype=torch.int32, device=DEV)
+        nk = torch.zeros(S, dtype=torch.int32, device=DEV)
+        g = torch.Generator().manual_seed(policy)
+        k = torch.randn(S, 2, cap, 64, generator=g).to(torch.bfloat16)
+        dk = k.to(DEV)
+        B.sirllm_keep_policy(cfg, policy, live, 1234567890123, 5, 10, keep, nk, ws)
+        B.sirllm_compact_kv(cfg, dk, None, dk, None, keep, nk, ws)
+        assert B.sirllm_status(ws) == 0
+        assert live.cpu().tolist() == lens
+        for s, l in enumerate(lens):
+            want = oracle.keep_policy(policy, l, n_sink, n_recent, budget, seed=1234567890123,
+                                      stream=10 + s, rnd=5)
+            n = int(nk[s])
+            assert n == len(want)
+            assert torch.equal(keep[s, :n].cpu(), want)
+            for p in range(2):
+                assert torch.equal(dk[s, p, :n].cpu(), oracle.gather_rows(k[s, p], want))
