@@ -423,3 +423,34 @@ def test_keep_policy_matches_oracle_and_feeds_the_gather(policy):
             assert torch.equal(keep[s, :n].cpu(), want)
             for p in range(2):
                 assert torch.equal(dk[s, p, :n].cpu(), oracle.gather_rows(k[s, p], want))
+
+
+def test_step_long_stream_without_reset_keeps_denormal_scores():
+    # The Rock-Paper-Scissors runs keep one cache for 2000 rounds of ~54 tokens (Table 7,
+    # Section 4.2.3) with 4 sinks + 1020 entropy slots and no recent window; here 2000 rounds at
+    # decay 0.7 on fewer planes.  The sink tokens are never evicted, so their scores decay through
+    # the denormal range and stick at the smallest denormal (0.7 * 2^-149 rounds back to 2^-149):
+    # flushing denormals to zero on the device would break bit parity here.
+    w = wl.WORKLOADS["rps_1024"].scaled(n_layers=1, n_kv_heads=2, vocab=2003, decay=0.7,
+                                        budget=260, capacity=320)
+    st = DeviceState(w)
+    tw = oracle_twin(w, st.decay.cpu(), with_kv=False)[0]
+    for r in range(2000):
+        st.fill_round(r)
+        st.step()
+        e = st.new_entropy[:w.new_tokens].cpu()
+        keep = tw.step(e)
+        n = tw.live_len
+        assert st.host_len == [n]
+        assert torch.equal(st.keep_idx[0, :n].cpu(), keep), r
+        assert torch.equal(st.scores[0, :n].cpu().view(torch.int32), tw.E[:n].view(torch.int32)), r
+        assert torch.equal(st.serial[0, :n].cpu(), tw.serial[:n]), r
+        if r % 200 == 199:
+            st.check_kv_by_content()
+            assert_entropy_close(e, oracle.score(st.logits[:w.new_tokens].cpu(), st.token_ids[:w.new_tokens].cpu()))
+    assert B.sirllm_status(st.ws) == 0
+    st.check_kv_by_content()
+    assert st.scores[0, :4].cpu().view(torch.int32).tolist() == [1, 1, 1, 1]     # 2^-149
+    # with decay < 1 nothing old survives (Appendix B): the cache holds only recent serials
+    newest = int(st.serial[0, :n].max())
+    assert int(st.serial[0, 4]) > newest - 40 * w.new_tokens
