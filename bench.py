@@ -235,10 +235,27 @@ def run_ours(args, rank, world, local_rank):
         p.step()
     sync()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    graph = None
+    if args.graph:       # two rounds (one per logits tensor) captured once, replayed K/2 times
+        assert args.steps % 2 == 0, "--graph needs an even --steps"
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                p.step()
+                p.step()
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay()
+        sync()
     with ClockSampler(local_rank) as clk:
         t0.record()
-        for _ in range(args.steps):
-            p.step()
+        if graph is None:
+            for _ in range(args.steps):
+                p.step()
+        else:
+            for _ in range(args.steps // 2):
+                graph.replay()
         t1.record()
         sync()
     ms_total = sharding.max_over_ranks(t0.elapsed_time(t1), dev)
@@ -287,7 +304,8 @@ def run_ours(args, rank, world, local_rank):
                            "planes": 2 * w.planes_per_stream, "head_dim": w.head_dim,
                            "capacity": w.capacity, "budget": w.budget, "n_sink": w.n_sink,
                            "n_recent": w.n_recent, "decay": w.decay, "parallelism": f"streams x{world}",
-                           "l2": "inputs larger than L2 (logits alternate between two tensors)"},
+                           "l2": "inputs larger than L2 (logits alternate between two tensors)",
+                           "cuda_graph": bool(args.graph)},
                 "clocks": clk.result, "e2e": e2e, "gpu_launches": 3 * args.steps,
                 "roofline": roofline}
         if cpu_baseline is not None:
@@ -452,6 +470,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(wl.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay the timed rounds from a captured CUDA graph (launch-bound shapes)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
