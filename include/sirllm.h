@@ -144,10 +144,9 @@ int sirllm_score_pairs(const sirllm_config *cfg, const void *pairs, int32_t n_ti
  * Same arguments and result as sirllm_score (scores are bit-identical), except:
  *   status   int32 device word that receives SIRLLM_STATUS_* bits (OR-ed in; the caller
  *            zeroes it), or NULL to drop them
- *   limits   n_streams * max_new <= 16384 rows, and rows * (CTAs per row) <= 65536, where a
- *            row takes ceil(vocab / 32768) CTAs for bf16 logits (vocab / 16384 for fp32) in
- *            large rounds and up to four times as many in small ones; beyond either limit
- *            SIRLLM_ERR_TOO_LARGE is returned and nothing runs
+ *   limits   n_streams * max_new <= 16384 rows, and rows * ceil(vocab / 32768 [bf16] or
+ *            16384 [fp32]) <= 65536; beyond that SIRLLM_ERR_TOO_LARGE is returned and
+ *            nothing runs
  * Things to know:
  *   - every GPU that loads the library holds the array until the process exits;
  *   - the first call on each device looks up the array's address on that device (the

@@ -40,13 +40,7 @@ WorkspaceLayout workspace_layout(const sirllm_config& c) {
     WorkspaceLayout L;
     const int64_t epv = 16 / logits_elem_bytes(c.logits_dtype);
     const int64_t nvec = c.vocab / epv;
-    // segment length: as long as possible while the scoring grid still has a few warps per
-    // scheduler on every SM (small rounds are latency bound otherwise)
-    const int64_t rows = (int64_t)c.n_streams * c.max_new;
-    int vps = kVecPerSegMax;
-    while (vps > kVecPerSegMin && rows * ((nvec + vps - 1) / vps) < 148 * 48) vps /= 2;
-    L.vec_per_seg = vps;
-    const int64_t per_cta = (int64_t)vps * kScoreWarpsPerCta;
+    const int64_t per_cta = (int64_t)kVecPerSeg * kScoreWarpsPerCta;
     L.n_part = (int32_t)((nvec + per_cta - 1) / per_cta);
     if (L.n_part < 1) L.n_part = 1;
     size_t off = 256;
@@ -90,7 +84,6 @@ static ScoreParams score_params(const sirllm_config& c, const WorkspaceLayout& L
     sp.n_streams = c.n_streams;
     sp.max_new = c.max_new;
     sp.n_part = L.n_part;
-    sp.vec_per_seg = L.vec_per_seg;
     sp.logits_dtype = c.logits_dtype;
     return sp;
 }

@@ -27,12 +27,10 @@ struct WorkspaceLayout {
     size_t policy_ones_off;
     size_t partials_off;
     size_t total;
-    int32_t n_part;       // CTAs (groups of kScoreWarpsPerCta segments) per logits row
-    int32_t vec_per_seg;  // 16-byte vectors one warp reduces
+    int32_t n_part;  // CTAs (groups of kScoreWarpsPerCta segments) per logits row
 };
 
-constexpr int kVecPerSegMax = 1024;  // 16-byte vectors per segment: at most 16 KB of logits per warp
-constexpr int kVecPerSegMin = 256;   // small problems use shorter segments to fill the GPU
+constexpr int kVecPerSeg = 1024;  // 16-byte vectors per segment: 16 KB of logits per warp
 constexpr int kScoreWarpsPerCta = 4;
 constexpr int kSelectThreads = 1024;
 constexpr int kRadixBits = 11;
@@ -56,7 +54,7 @@ struct ScoreParams {
     const int32_t* live_len;   // with `scores`
     int64_t vocab;
     int64_t row_stride;
-    int32_t n_streams, max_new, n_part, vec_per_seg, logits_dtype, capacity;
+    int32_t n_streams, max_new, n_part, logits_dtype, capacity;
 };
 
 struct PairScoreParams {

@@ -1,9 +1,9 @@
 // Token Entropy (Section 3.2): e = -log softmax(z)[id] as a vocabulary-streaming
-// log-sum-exp.  Every logits row is cut into segments of 256..1024 16-byte vectors;
+// log-sum-exp.  Every logits row is cut into segments of kVecPerSeg 16-byte vectors;
 // one warp reduces one segment with an online (running-max) softmax sum, and the
 // kScoreWarpsPerCta warps of a CTA (consecutive segments of one row) combine their
-// (scaled max, sum) pairs through shared memory.  A row that needs several CTAs (more
-// than 4 segments) publishes one pair per CTA in
+// (scaled max, sum) pairs through shared memory.  A row that needs several CTAs
+// (vocabularies above 32768 bf16 / 16384 fp32 elements) publishes one pair per CTA in
 // scratch; the CTA that arrives last on the row's ticket combines them.  Combination is
 // in fp64 and in a fixed order, so the score does not depend on which CTA comes last.
 // The finishing warp writes the score and, in the fused round, appends it to E.
@@ -87,8 +87,8 @@ score_kernel(const ScoreParams p) {
     const int64_t nvec = (V - head) / EPV;
     const int64_t tail = V - head - nvec * EPV;
     const uint4* vec = (const uint4*)(rowp + head * ES);
-    const int64_t v0 = (int64_t)seg * p.vec_per_seg;
-    const int64_t v1 = min(v0 + (int64_t)p.vec_per_seg, nvec);
+    const int64_t v0 = (int64_t)seg * kVecPerSeg;
+    const int64_t v1 = min(v0 + (int64_t)kVecPerSeg, nvec);
     const uint32_t neg_inf = kBf16 ? 0xFF80FF80u : 0xFF800000u;
 
     // software pipeline: the loads of trip i+1 are in flight while trip i is reduced
@@ -361,7 +361,6 @@ extern "C" int sirllm_score_static(const sirllm_config* cfg, const void* logits,
     sp.n_streams = cfg->n_streams;
     sp.max_new = cfg->max_new;
     sp.n_part = L.n_part;
-    sp.vec_per_seg = L.vec_per_seg;
     sp.logits_dtype = cfg->logits_dtype;
     sp.capacity = cfg->capacity;
     e = launch_score(sp, st);
