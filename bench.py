@@ -208,6 +208,17 @@ def step_bytes(w: wl.Workload, moved_rows: int) -> dict:
     return {"score": score, "select": select, "compact": compact, "step": score + select + compact}
 
 
+def config_dict(w: wl.Workload, world: int, graph: bool = False) -> dict:
+    return {"workload": w.name, "streams_per_gpu": w.n_streams,
+            "new_tokens_per_round": w.new_tokens, "vocab": w.vocab,
+            "logits_dtype": w.logits_dtype, "kv_dtype": w.kv_dtype,
+            "planes": 2 * w.planes_per_stream, "head_dim": w.head_dim,
+            "capacity": w.capacity, "budget": w.budget, "n_sink": w.n_sink,
+            "n_recent": w.n_recent, "decay": w.decay, "parallelism": f"streams x{world}",
+            "l2": "inputs larger than L2 (logits alternate between two tensors)",
+            "cuda_graph": graph}
+
+
 def run_ours(args, rank, world, local_rank):
     from paper_2405_12528_b200 import binding as B
     B.lib()                                       # fail loudly if the CUDA library is missing
@@ -298,14 +309,7 @@ def run_ours(args, rank, world, local_rank):
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_step, 4),
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "f32", "data": "synthetic",
-                "config": {"workload": w.name, "streams_per_gpu": w.n_streams,
-                           "new_tokens_per_round": w.new_tokens, "vocab": w.vocab,
-                           "logits_dtype": w.logits_dtype, "kv_dtype": w.kv_dtype,
-                           "planes": 2 * w.planes_per_stream, "head_dim": w.head_dim,
-                           "capacity": w.capacity, "budget": w.budget, "n_sink": w.n_sink,
-                           "n_recent": w.n_recent, "decay": w.decay, "parallelism": f"streams x{world}",
-                           "l2": "inputs larger than L2 (logits alternate between two tensors)",
-                           "cuda_graph": bool(args.graph)},
+                "config": config_dict(w, world, bool(args.graph)),
                 "clocks": clk.result, "e2e": e2e, "gpu_launches": 3 * args.steps,
                 "roofline": roofline}
         if cpu_baseline is not None:
@@ -454,7 +458,7 @@ def run_reference(args, rank, world):
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name},
+            "config": config_dict(w, world),
             "cpu_baseline": {"value": round(value, 1), "unit": UNIT, "cores": 1, "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": round(value, 1), "unit": UNIT, "h2d_bytes_per_step": 0,

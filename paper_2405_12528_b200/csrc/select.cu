@@ -65,6 +65,7 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     if (blockIdx.x == 0 && tid == 0) *p.epoch += 1;  // a new compaction follows
 
     const int l0 = p.live_len[s];
+    const float eta = p.decay[s];  // fetched together with the lengths: one round trip
     int T = 0;
     if (p.score_new) {  // the scorer has appended T raw scores behind slot l0
         T = p.n_new ? p.n_new[s] : p.max_new;
@@ -82,13 +83,27 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     const int l = l0 + T;
 
     // ---- S3: one fp32 multiply per held score -----------------------------------------
-    const float eta = p.decay[s];
     const bool evict = l > p.threshold;
     const bool write_now = !(evict && p.compact_scores);
-    for (int i = tid; i < l; i += kSelectThreads) {
-        const float x = __fmul_rn(scores[i], eta);
-        vals[i] = __float_as_uint(x);
-        if (write_now) scores[i] = x;
+    // loads are issued in batches before any of them is used, so the block pays one memory
+    // round trip per batch instead of one per element
+    constexpr int kLoadBatch = 16;
+    for (int base = 0; base < l; base += kLoadBatch * kSelectThreads) {
+        float x[kLoadBatch];
+#pragma unroll
+        for (int q = 0; q < kLoadBatch; ++q) {
+            const int i = base + q * kSelectThreads + tid;
+            x[q] = i < l ? scores[i] : 0.f;
+        }
+#pragma unroll
+        for (int q = 0; q < kLoadBatch; ++q) {
+            const int i = base + q * kSelectThreads + tid;
+            if (i < l) {
+                const float v = __fmul_rn(x[q], eta);
+                vals[i] = __float_as_uint(v);
+                if (write_now) scores[i] = v;
+            }
+        }
     }
     if (!evict) {  // ---- nothing to evict: identity keep list --------------------------
         for (int i = tid; i < l; i += kSelectThreads) keep[i] = i;
