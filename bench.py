@@ -42,11 +42,10 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from one ncu capture (profiles/compact_kernel_*.md):
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch on the small profiling case.
 # Traffic grows in proportion to the moved bytes, so it is scaled to the timed launch; it
-# is reported only while the kernel's sources are the ones the counters were taken on.
+# is reported only while the kernel's source file is the one the counters were taken on.
 NCU_CAPTURE = {"kernel": "compact_kernel", "workload": "llama3_8b_quarter",
                "dram_bytes": 267954688 + 214801920, "algorithmic_bytes": 2 * 2044 * 256 * 512,
-               "sources": {"paper_2405_12528_b200/csrc/compact.cu": "5a73a5c0abc81843c030398e7e68774a28b94481",
-                           "paper_2405_12528_b200/csrc/common.cuh": "2d7831351ca583eff4dd5eeda078a670e52ce9cd"}}
+               "sources": {"paper_2405_12528_b200/csrc/compact.cu": "5a73a5c0abc81843c030398e7e68774a28b94481"}}
 
 
 def ncu_traffic(bytes_per_launch):
