@@ -32,9 +32,7 @@ struct WorkspaceLayout {
 
 constexpr int kVecPerSeg = 1024;  // 16-byte vectors per segment: 16 KB of logits per warp
 constexpr int kScoreWarpsPerCta = 4;
-constexpr int kSelectThreads = 1024;
-constexpr int kRadixBits = 11;
-constexpr int kRadixBins = 1 << kRadixBits;
+constexpr int kListMax = 256;  // keys ranked directly once a radix bin holds no more
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int logits_elem_bytes(int dtype) { return dtype == SIRLLM_F32 ? 4 : 2; }

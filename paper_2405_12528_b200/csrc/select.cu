@@ -2,26 +2,39 @@
 // (Section 3.3: E = E x eta_decay, Top_k(E); Section 3.1: sink and recent sets;
 // Algorithm 1: the test "cache size > L").
 //
-// All scores of the stream live in shared memory as fp32 bit patterns.  The k-th
-// largest middle score is found by a most-significant-digit radix select on the
-// order-preserving key (11-bit digits, skipping the bits all keys share), ties at the
-// threshold are resolved towards the lower slot, and the keep list is emitted in
-// ascending order with warp ballots and a block prefix sum.  Touches at most a few
-// hundred KB: this is the latency-bound serial link between scoring and KV compaction.
+// All scores of the stream live in shared memory as fp32 bit patterns.  The k-th largest
+// middle score is found on the order-preserving integer key of the bit pattern:
+//   1. min and max key of the middle slots (block reduction);
+//   2. a most-significant-digit radix pass over d = key - min (11-bit digits of the range the
+//      keys really span, 2048-bin shared histogram, block scan from the top bin);
+//   3. as soon as the bin that holds the k-th key has at most kListMax members they are listed
+//      and ranked directly; otherwise the next digit is taken (ties in bulk, tiny ranges).
+// Ties at the threshold are resolved towards the lower slot.  The ascending keep list and the
+// compacted scores are then written by threads that each own a contiguous run of slots (count,
+// block prefix sum, write), and the 8-byte tags follow in register batches.
+// The kernel runs on one SM and touches at most a few hundred KB: it is the instruction- and
+// latency-bound serial link between scoring and KV compaction.
 #include "common.cuh"
 
 namespace sirllm {
 
 namespace {
 
+constexpr int kSelectThreads = 1024;
+constexpr int kRadixBits = 11;
+constexpr int kRadixBins = 1 << kRadixBits;
+constexpr int kListMax = 256;  // keys ranked directly once the radix bin holds no more
+
 struct BlockScratch {
     int warp_sum[32];
-    int warp_sure[32];
-    int warp_eq[32];
-    uint32_t red_and[32];
-    uint32_t red_or[32];
+    uint32_t red_min[32];
+    uint32_t red_max[32];
     int bin;
     int above;
+    int bin_count;
+    int list_n;
+    uint32_t tau;
+    int r;
     int first_evicted;
 };
 
@@ -49,10 +62,15 @@ __device__ __forceinline__ int block_inclusive_scan(int v, int* warp_sum) {
     return v;
 }
 
+// kStage: the keep list is assembled in shared memory and written out coalesced (the host
+// chooses this whenever capacity + threshold words fit); otherwise it goes straight to global
+// memory from the owning threads.
+template <bool kStage>
 __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectParams p) {
-    extern __shared__ uint32_t smem[];
-    uint32_t* vals = smem;                        // [capacity] fp32 bit patterns
-    int* hist = (int*)(smem + p.capacity);        // [kRadixBins]
+    extern __shared__ __align__(16) uint32_t smem[];
+    uint32_t* vals = smem;                                      // [capacity] fp32 bit patterns
+    int* hist = (int*)(smem + ((p.capacity + 3) & ~3) + 4);     // [kRadixBins]
+    int* skeep = hist + kRadixBins;                             // [threshold] when kStage
     __shared__ BlockScratch sh;
 
     const int s = blockIdx.x;
@@ -88,6 +106,8 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     // loads are issued in batches before any of them is used, so the block pays one memory
     // round trip per batch instead of one per element
     constexpr int kLoadBatch = 16;
+    const int lo = p.n_sink, hi = l - p.n_recent;
+    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;  // over the middle slots' keys (for S4)
     for (int base = 0; base < l; base += kLoadBatch * kSelectThreads) {
         float x[kLoadBatch];
 #pragma unroll
@@ -102,6 +122,11 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
                 const float v = __fmul_rn(x[q], eta);
                 vals[i] = __float_as_uint(v);
                 if (write_now) scores[i] = v;
+                if (i >= lo && i < hi) {
+                    const uint32_t key = order_key(__float_as_uint(v));
+                    kmin = min(kmin, key);
+                    kmax = max(kmax, key);
+                }
             }
         }
     }
@@ -114,40 +139,33 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
         }
         return;
     }
-    __syncthreads();
 
     // ---- S4: threshold key of the top-k among the middle slots ---------------------------
-    const int lo = p.n_sink, hi = l - p.n_recent;
     const int k = p.budget - p.n_sink - p.n_recent;
     uint32_t tau = 0xFFFFFFFFu;  // with k == 0 nothing in the middle is kept
     int r = 0;                   // how many slots with key == tau are kept (lowest slots first)
     if (k > 0) {
-        uint32_t a = 0xFFFFFFFFu, o = 0u;
-        for (int i = lo + tid; i < hi; i += kSelectThreads) {
-            const uint32_t key = order_key(vals[i]);
-            a &= key;
-            o |= key;
-        }
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) {
-            a &= __shfl_xor_sync(0xFFFFFFFFu, a, d);
-            o |= __shfl_xor_sync(0xFFFFFFFFu, o, d);
+            kmin = min(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, d));
+            kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, d));
         }
         if (lane == 0) {
-            sh.red_and[wid] = a;
-            sh.red_or[wid] = o;
+            sh.red_min[wid] = kmin;
+            sh.red_max[wid] = kmax;
         }
-        __syncthreads();
-        a = sh.red_and[lane];
-        o = sh.red_or[lane];
+        __syncthreads();  // also orders the writes of vals before the reads below
+        kmin = sh.red_min[lane];
+        kmax = sh.red_max[lane];
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) {
-            a &= __shfl_xor_sync(0xFFFFFFFFu, a, d);
-            o |= __shfl_xor_sync(0xFFFFFFFFu, o, d);
+            kmin = min(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, d));
+            kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, d));
         }
-        const uint32_t diff = a ^ o;
-        int undecided = diff ? 32 - __clz(diff) : 0;  // low bits not yet fixed
-        uint32_t prefix = undecided < 32 ? (a >> undecided) : 0u;  // the shared high bits
+        // from here on keys are taken relative to the smallest one: d = key - kmin < 2^undecided
+        const uint32_t range = kmax - kmin;
+        int undecided = range ? 32 - __clz(range) : 0;  // low bits of d not yet fixed
+        uint32_t prefix = 0u;                           // the fixed high bits of d
         int need = k;
         while (undecided > 0) {
             const int w = min(kRadixBits, undecided);
@@ -155,9 +173,9 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
             for (int b = tid; b < kRadixBins; b += kSelectThreads) hist[b] = 0;
             __syncthreads();
             for (int i = lo + tid; i < hi; i += kSelectThreads) {
-                const uint32_t key = order_key(vals[i]);
-                if ((uint32_t)((uint64_t)key >> undecided) == prefix)
-                    atomicAdd(&hist[(key >> sh_amt) & ((1u << w) - 1u)], 1);
+                const uint32_t d = order_key(vals[i]) - kmin;
+                if ((uint32_t)((uint64_t)d >> undecided) == prefix)
+                    atomicAdd(&hist[(d >> sh_amt) & ((1u << w) - 1u)], 1);
             }
             __syncthreads();
             // walk the bins from the largest digit down; thread t owns two of them
@@ -168,82 +186,127 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
             if (excl < need && need <= excl + c0) {
                 sh.bin = kRadixBins - 1 - 2 * tid;
                 sh.above = excl;
+                sh.bin_count = c0;
+                sh.list_n = 0;
             } else if (excl + c0 < need && need <= incl) {
                 sh.bin = kRadixBins - 2 - 2 * tid;
                 sh.above = excl + c0;
+                sh.bin_count = c1;
+                sh.list_n = 0;
             }
             __syncthreads();
             prefix = (prefix << w) | (uint32_t)sh.bin;
             need -= sh.above;
             undecided = sh_amt;
+            const int n_left = sh.bin_count;
             __syncthreads();
+            if (undecided > 0 && n_left <= kListMax) {
+                // few keys are left in the bin: list them and rank them directly instead of
+                // running the remaining digit passes
+                uint32_t* list = reinterpret_cast<uint32_t*>(hist);
+                for (int i = lo + tid; i < hi; i += kSelectThreads) {
+                    const uint32_t d = order_key(vals[i]) - kmin;
+                    if ((d >> undecided) == prefix) list[atomicAdd(&sh.list_n, 1)] = d;
+                }
+                __syncthreads();
+                if (tid < n_left) {
+                    const uint32_t mine = list[tid];
+                    int greater = 0, equal = 0;
+                    for (int j = 0; j < n_left; ++j) {
+                        const uint32_t other = list[j];
+                        greater += other > mine;
+                        equal += other == mine;
+                    }
+                    if (greater < need && need <= greater + equal) {  // the need-th largest
+                        sh.tau = mine;
+                        sh.r = need - greater;
+                    }
+                }
+                __syncthreads();
+                prefix = sh.tau;
+                need = sh.r;
+                undecided = 0;
+            }
         }
-        tau = prefix;
+        tau = kmin + prefix;
         r = need;
+    } else {
+        __syncthreads();  // vals complete
     }
 
     // ---- S4 (emit) + S5: ascending keep list, compacted scores ------------------------------
-    // warp w owns a contiguous span of slots; sure = sink / recent / above the threshold key
-    const int span = ((l + 31) / 32 + 31) & ~31;
-    const int w_begin = wid * span, w_end = min(l, w_begin + span);
+    // every thread owns a contiguous run of slots (a multiple of 4, read as 128-bit vectors);
+    // sure = sink / recent / above the threshold key, eq = at the threshold key
+    const int run = ((l + kSelectThreads - 1) / kSelectThreads + 3) & ~3;
+    const int i0 = min(l, tid * run), i1 = min(l, i0 + run);
     int n_sure = 0, n_eq = 0;
-    for (int base = w_begin; base < w_end; base += 32) {
-        const int i = base + lane;
-        bool sure = false, eq = false;
-        if (i < w_end) {
-            if (i < lo || i >= hi) {
-                sure = true;
-            } else {
-                const uint32_t key = order_key(vals[i]);
-                sure = key > tau;
-                eq = key == tau;
+    for (int i = i0; i < i1; i += 4) {
+        const uint4 q = *reinterpret_cast<const uint4*>(vals + i);  // beyond l: stale, masked
+        const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int j = i + c;
+            if (j < i1) {
+                if (j < lo || j >= hi) {
+                    ++n_sure;
+                } else {
+                    const uint32_t key = order_key(w4[c]);
+                    n_sure += key > tau;
+                    n_eq += key == tau;
+                }
             }
         }
-        n_sure += __popc(__ballot_sync(0xFFFFFFFFu, sure));
-        n_eq += __popc(__ballot_sync(0xFFFFFFFFu, eq));
     }
     if (tid == 0) sh.first_evicted = l;
-    if (lane == 0) {
-        sh.warp_sure[wid] = n_sure;
-        sh.warp_eq[wid] = n_eq;
-    }
-    __syncthreads();
-    int sure_before = 0, eq_before = 0;
-    for (int q = 0; q < wid; ++q) {
-        sure_before += sh.warp_sure[q];
-        eq_before += sh.warp_eq[q];
-    }
-    int kept_before = sure_before + min(eq_before, r);
-    const uint32_t lt_mask = (1u << lane) - 1u;
-    for (int base = w_begin; base < w_end; base += 32) {
-        const int i = base + lane;
-        bool sure = false, eq = false;
-        uint32_t bits = 0;
-        if (i < w_end) {
-            bits = vals[i];
-            if (i < lo || i >= hi) {
-                sure = true;
-            } else {
-                const uint32_t key = order_key(bits);
-                sure = key > tau;
-                eq = key == tau;
+    // both counts are at most 49152 < 2^16: one packed scan
+    const int packed = n_sure | (n_eq << 16);
+    const int before = block_inclusive_scan(packed, sh.warp_sum) - packed;
+    int eq_before = (int)((uint32_t)before >> 16);
+    int pos = (before & 0xFFFF) + min(eq_before, r);
+    int my_first_evicted = l;
+    for (int i = i0; i < i1; i += 4) {
+        const uint4 q = *reinterpret_cast<const uint4*>(vals + i);
+        const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int j = i + c;
+            if (j < i1) {
+                bool kept = true;
+                if (j >= lo && j < hi) {
+                    const uint32_t key = order_key(w4[c]);
+                    kept = key > tau;
+                    if (key == tau) {
+                        kept = eq_before < r;
+                        ++eq_before;
+                    }
+                }
+                if (kept) {
+                    if (kStage) {
+                        skeep[pos] = j;
+                    } else {
+                        keep[pos] = j;
+                        if (p.compact_scores) scores[pos] = __uint_as_float(w4[c]);
+                    }
+                    ++pos;
+                } else {
+                    my_first_evicted = min(my_first_evicted, j);
+                }
             }
         }
-        const uint32_t eq_ballot = __ballot_sync(0xFFFFFFFFu, eq);
-        const bool kept = sure || (eq && eq_before + __popc(eq_ballot & lt_mask) < r);
-        const uint32_t kept_ballot = __ballot_sync(0xFFFFFFFFu, kept);
-        if (kept) {
-            const int pos = kept_before + __popc(kept_ballot & lt_mask);
-            keep[pos] = i;
-            if (p.compact_scores) scores[pos] = __uint_as_float(bits);
-        } else if (i < w_end) {
-            atomicMin(&sh.first_evicted, i);
-        }
-        kept_before += __popc(kept_ballot);
-        eq_before += __popc(eq_ballot);
     }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1)
+        my_first_evicted = min(my_first_evicted, __shfl_xor_sync(0xFFFFFFFFu, my_first_evicted, d));
+    if (lane == 0 && my_first_evicted < l) atomicMin(&sh.first_evicted, my_first_evicted);
     __syncthreads();
     const int first = sh.first_evicted;
+    if (kStage) {  // coalesced copy-out of the list and of the scores it selects
+        for (int j = tid; j < p.budget; j += kSelectThreads) {
+            const int src = skeep[j];
+            keep[j] = src;
+            if (p.compact_scores) scores[j] = __uint_as_float(vals[src]);
+        }
+    }
 
     // ---- S5: the 8-byte tags follow, in place, front to back.  A batch of kTagBatch tags
     // per thread is read into registers before any of them is written; a later batch only
@@ -256,7 +319,7 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
 #pragma unroll
             for (int q = 0; q < kTagBatch; ++q) {
                 const int j = base + q * kSelectThreads + tid;
-                v[q] = j < p.budget ? serial[keep[j]] : 0;
+                v[q] = j < p.budget ? serial[kStage ? skeep[j] : keep[j]] : 0;
             }
             __syncthreads();
 #pragma unroll
@@ -277,9 +340,18 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
 }  // namespace
 
 cudaError_t launch_select(const SelectParams& p, int n_streams, cudaStream_t st, bool overlap) {
-    const size_t smem = (size_t)p.capacity * 4 + (size_t)kRadixBins * 4;
-    cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    // scores (rounded up to whole 128-bit vectors, plus one vector of slack) + histogram
+    // (+ the staged keep list when it fits)
+    size_t smem = ((size_t)((p.capacity + 3) & ~3) + 4) * 4 + (size_t)kRadixBins * 4;
+    int dev = 0, smem_max = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) return e;
+    const bool stage = smem + (size_t)p.threshold * 4 + 1024 <= (size_t)smem_max;
+    if (stage) smem += (size_t)p.threshold * 4;
+    auto kernel = stage ? select_kernel<true> : select_kernel<false>;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)n_streams);
@@ -291,7 +363,7 @@ cudaError_t launch_select(const SelectParams& p, int n_streams, cudaStream_t st,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, select_kernel, p);
+    return cudaLaunchKernelEx(&cfg, kernel, p);
 }
 
 }  // namespace sirllm
