@@ -65,12 +65,14 @@ extern "C" {
 /* Largest `capacity` the selection kernel supports (the scores of one stream are
  * held in one SM's shared memory). */
 #define SIRLLM_MAX_CAPACITY 49152
+/* Largest `head_dim` (K/V rows of at most 1 KB; the gather stages 32 rows per copy). */
+#define SIRLLM_MAX_HEAD_DIM 512
 
 typedef struct sirllm_config {
     int32_t n_streams;   /* independent dialogue streams, >= 1 */
     int32_t n_layers;    /* K/V planes per stream = n_layers * n_kv_heads (each of K and V) */
     int32_t n_kv_heads;
-    int32_t head_dim;    /* elements per K/V row; head_dim * 2 bytes must be a multiple of 16 */
+    int32_t head_dim;    /* elements per K/V row, a multiple of 8, <= SIRLLM_MAX_HEAD_DIM */
     int32_t capacity;    /* physical slots per plane, <= SIRLLM_MAX_CAPACITY */
     int32_t budget;      /* retained slots after an eviction = n_sink + n_recent + k  (the
                             "cache size" of Tables 1-3) */

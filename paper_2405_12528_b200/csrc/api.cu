@@ -29,7 +29,7 @@ int validate_config(const sirllm_config* c) {
         return SIRLLM_ERR_BAD_CONFIG;
     if (c->vocab < 1 || c->vocab > 0x7FFFFFFF || c->logits_row_stride < c->vocab)
         return SIRLLM_ERR_BAD_CONFIG;
-    if ((int64_t)c->head_dim * 2 % 16 != 0 || (int64_t)c->head_dim * 2 > 4096)
+    if ((int64_t)c->head_dim * 2 % 16 != 0 || c->head_dim > SIRLLM_MAX_HEAD_DIM)
         return SIRLLM_ERR_BAD_CONFIG;
     if ((int64_t)c->n_streams * c->n_layers * c->n_kv_heads > 0x3FFFFFFF)
         return SIRLLM_ERR_BAD_CONFIG;

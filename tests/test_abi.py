@@ -42,7 +42,7 @@ def test_workspace_size_is_pure_and_zero_for_bad_configs(lib):
     n = B.sirllm_workspace_bytes(_cfg())
     assert n > 0 and n % 256 == 0 and n == B.sirllm_workspace_bytes(_cfg())
     assert B.sirllm_workspace_bytes(_cfg(max_new=1024)) > n
-    for bad in (dict(budget=60), dict(threshold=100), dict(capacity=200), dict(head_dim=12),
+    for bad in (dict(budget=60), dict(threshold=100), dict(capacity=200), dict(head_dim=12), dict(head_dim=520),
                 dict(capacity=B.MAX_CAPACITY + 1), dict(n_streams=0), dict(vocab=0),
                 dict(logits_row_stride=31999), dict(logits_dtype="f16"), dict(kv_dtype="f32"),
                 dict(n_sink=-1)):

@@ -227,6 +227,8 @@ def test_compact_matches_gather(in_place):
     _compact_case(1, 3, 1000, 64, [999], in_place, 1, torch.float16)       # ragged last chunk
     _compact_case(3, 2, 64, 8, [0, 1, 64], in_place, 2)                    # empty, single, full
     _compact_case(1, 700, 96, 128, [50], in_place, 3)                      # more planes than workers
+    _compact_case(1, 6, 400, 256, [333], in_place, 4)                      # 512-byte rows
+    _compact_case(2, 3, 200, 512, [150, 199], in_place, 5)                 # 1 KB rows: the largest
 
 
 def test_compact_identity_list_moves_nothing_and_bad_lists_are_refused():
