@@ -200,7 +200,10 @@ __device__ __forceinline__ void bulk_wait_read() {
 __device__ __forceinline__ void bulk_wait_all() {
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
-constexpr uint32_t kSpinLimit = 1u << 22;  // polls before a device-side wait gives up
+// polls before a device-side wait gives up (a healthy wait ends within microseconds for an
+// mbarrier and within one kernel duration for a progress word; these limits are seconds)
+constexpr uint32_t kSpinLimit = 1u << 22;      // global-memory progress words
+constexpr uint32_t kMbarSpinLimit = 1u << 20;  // mbarrier phases (each poll may itself suspend)
 
 // Order-preserving map from fp32 bit patterns to unsigned integers: a larger key is a
 // larger score; negatives sort below non-negatives and -0 below +0.

@@ -61,7 +61,7 @@ __device__ __forceinline__ bool store_chunk(uint64_t* full, StageInfo* info, cha
     if (lane == 0) {
         const int stage = (int)(c % stages);
         const uint32_t parity = (uint32_t)((c / stages) & 1);
-        ok = mbar_wait_bounded(&full[stage], parity, kSpinLimit);
+        ok = mbar_wait_bounded(&full[stage], parity, kMbarSpinLimit);
         const StageInfo si = info[stage];
         if (ok && si.wait_val != 0) {
             uint32_t spins = 0;
