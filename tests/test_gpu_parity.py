@@ -456,3 +456,62 @@ def test_step_long_stream_without_reset_keeps_denormal_scores():
     # with decay < 1 nothing old survives (Appendix B): the cache holds only recent serials
     newest = int(st.serial[0, :n].max())
     assert int(st.serial[0, 4]) > newest - 40 * w.new_tokens
+
+
+def test_select_randomised_shapes_and_score_patterns():
+    # many seeded draws of (lengths, sinks, recent, budget, threshold, decay) and of score
+    # patterns that steer the selection kernel through all its branches: narrow key ranges (one
+    # short digit), bulk ties (several digit passes), few distinct values, negative and zero
+    # scores, k = 1 and k = all-but-one
+    rng = np.random.default_rng(12345)
+    for case in range(60):
+        cap = int(rng.choice([64, 300, 1000, 4096, 9000]))
+        n_sink = int(rng.integers(0, 6))
+        n_recent = int(rng.integers(0, max(1, cap // 8)))
+        k = int(rng.choice([0, 1, 2, int(rng.integers(1, max(2, cap // 2)))]))
+        budget = max(1, n_sink + n_recent + k)
+        if budget > cap:
+            continue
+        threshold = int(min(cap, budget + rng.choice([0, 0, 3, cap // 10])))
+        S = int(rng.integers(1, 5))
+        lens = [int(rng.integers(0, cap + 1)) for _ in range(S)]
+        lens[0] = int(min(cap, budget + 1 + rng.integers(0, max(1, cap - budget))))   # evicts
+        if rng.random() < 0.3:
+            lens[-1] = min(cap, threshold + 1)                                          # evicts one
+        cfg = B.make_config(S, 1, 1, 8, cap, budget, n_sink, n_recent, 0, 16, torch.float32,
+                            torch.bfloat16, threshold=threshold)
+        ws = B.new_workspace(cfg)
+        E = torch.zeros(S, cap)
+        pattern = case % 6
+        for s, l in enumerate(lens):
+            u = torch.tensor(rng.random(l), dtype=torch.float32)
+            if pattern == 0:
+                E[s, :l] = u * 12
+            elif pattern == 1:
+                E[s, :l] = 3.0 + u * 1e-5                      # narrow range
+            elif pattern == 2:
+                E[s, :l] = torch.round(u * 3)                  # 4 distinct values: bulk ties
+            elif pattern == 3:
+                E[s, :l] = (u - 0.5) * 4                       # negatives too
+            elif pattern == 4:
+                E[s, :l] = torch.where(u < 0.7, torch.zeros(()), u)   # mostly exact zeros
+            else:
+                E[s, :l] = torch.exp((u - 0.5) * 60)           # 26 orders of magnitude
+        decay = [float(rng.choice([1.0, 0.9, 0.5])) for _ in range(S)]
+        serial = torch.arange(S * cap, dtype=torch.int64).view(S, cap)
+        dE, dser = E.to(DEV), serial.to(DEV)
+        dlen = torch.tensor(lens, dtype=torch.int32, device=DEV)
+        keep = torch.full((S, threshold), -1, dtype=torch.int32, device=DEV)
+        nk = torch.zeros(S, dtype=torch.int32, device=DEV)
+        B.sirllm_decay_select(cfg, dE, dser, dlen, torch.tensor(decay, device=DEV), keep, nk, 1, ws)
+        assert B.sirllm_status(ws) == 0
+        for s, l in enumerate(lens):
+            Es = E[s].clone()
+            oracle.decay(Es, l, decay[s])
+            want = oracle.select(Es, l, n_sink, n_recent, budget, threshold)
+            n = int(nk[s])
+            ctx = (case, s, l, n_sink, n_recent, budget, threshold, pattern)
+            assert n == len(want) == int(dlen[s]), ctx
+            assert torch.equal(keep[s, :n].cpu(), want), ctx
+            assert torch.equal(dE[s, :n].cpu().view(torch.int32), Es[want.long()].view(torch.int32)), ctx
+            assert torch.equal(dser[s, :n].cpu(), serial[s][want.long()]), ctx
