@@ -301,6 +301,7 @@ def run_ours(args, rank, world, local_rank):
                 "step_frac": round(by["step"] / (ms_step * 1e-3) / 1e9 / peak, 4),
                 "step_frac_of_8000": round(by["step"] / (ms_step * 1e-3) / 1e9 / 8000.0, 4)}
 
+    extras = run_extras(p, args) if args.extras else None
     e2e = run_e2e(p, args, dist, world)
 
     if rank == 0:
@@ -313,9 +314,65 @@ def run_ours(args, rank, world, local_rank):
                 "roofline": roofline}
         if cpu_baseline is not None:
             line["cpu_baseline"] = cpu_baseline
+        if extras is not None:
+            line["extras"] = extras
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def _time_rounds(fn, n):
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(n):
+        fn()
+    t1.record()
+    torch.cuda.synchronize()
+    return t0.elapsed_time(t1) / n
+
+
+def run_extras(p: Pass, args):
+    """Timings of the widened entry points on the same state: the fused round fed by per-tile
+    (max, sum-exp) pairs instead of logits, and the comparison policies' keep lists + gather."""
+    w, B, cfg = p.w, p.B, p.cfg
+    tile = 128
+    n_tiles = (w.vocab + tile - 1) // tile
+    pools = []
+    for lg, ids in p.pool:                       # what an LM-head epilogue would hand over
+        rows = lg.shape[0]
+        pairs = torch.empty(rows, n_tiles, 2, dtype=torch.float32, device=p.dev)
+        for r0 in range(0, rows, 512):
+            z = torch.full((min(512, rows - r0), n_tiles * tile), float("-inf"), device=p.dev)
+            z[:, :w.vocab] = lg[r0:r0 + 512].float()
+            z = z.view(-1, n_tiles, tile)
+            m = z.max(dim=2).values
+            pairs[r0:r0 + 512, :, 0] = m
+            pairs[r0:r0 + 512, :, 1] = torch.exp(z - m[:, :, None]).sum(dim=2)
+        target = lg.float()[torch.arange(rows, device=p.dev), ids.long()].contiguous()
+        pools.append((pairs, target, ids))
+    state = {"i": 0}
+
+    def pairs_round():
+        pairs, target, ids = pools[state["i"] & 1]
+        state["i"] += 1
+        B.sirllm_step_pairs(cfg, pairs, target, ids, p.n_new, p.scores, p.serial, p.live_len, p.decay,
+                            p.k, p.v, p.keep_idx, p.n_keep, p.new_entropy, p.ws)
+
+    out = {"pairs_tile": tile,
+           "step_pairs_ms": round(_time_rounds(pairs_round, args.steps), 4)}
+    full = torch.full_like(p.live_len, w.budget + w.new_tokens)
+    for name, pol in (("stream", B.POLICY_STREAM), ("random", B.POLICY_RANDOM), ("interval", B.POLICY_INTERVAL)):
+        def policy_round():
+            state["i"] += 1
+            B.sirllm_keep_policy(cfg, pol, full, 7, state["i"], 0, p.keep_idx, p.n_keep, p.ws)
+            B.sirllm_compact_kv(cfg, p.k, p.v, p.k, p.v, p.keep_idx, p.n_keep, p.ws)
+        out[f"policy_{name}_ms"] = round(_time_rounds(policy_round, args.steps), 4)
+    assert B.sirllm_status(p.ws) == 0
+    p.live_len.fill_(w.budget)
+    return out
 
 
 def run_e2e(p: Pass, args, dist, world):
@@ -473,6 +530,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(wl.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--extras", action="store_true",
+                    help="also time the pairs-fed round and the comparison policies")
     ap.add_argument("--graph", action="store_true",
                     help="replay the timed rounds from a captured CUDA graph (launch-bound shapes)")
     args = ap.parse_args()
