@@ -9,7 +9,7 @@ namespace sirllm {
 
 static thread_local char g_cuda_msg[256] = "";
 
-static int cuda_fail(cudaError_t e, const char* where) {
+int cuda_fail(cudaError_t e, const char* where) {
     snprintf(g_cuda_msg, sizeof g_cuda_msg, "%s: %s", where, cudaGetErrorString(e));
     return SIRLLM_ERR_CUDA;
 }

@@ -38,6 +38,8 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int logits_elem_bytes(int dtype) { return dtype == SIRLLM_F32 ? 4 : 2; }
 
 int validate_config(const sirllm_config* cfg);
+// Records the message sirllm_last_cuda_error() returns and yields SIRLLM_ERR_CUDA.
+int cuda_fail(cudaError_t e, const char* where);
 WorkspaceLayout workspace_layout(const sirllm_config& cfg);
 
 struct ScoreParams {

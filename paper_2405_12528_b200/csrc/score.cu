@@ -341,11 +341,11 @@ extern "C" int sirllm_score_static(const sirllm_config* cfg, const void* logits,
     if (rows == 0) return SIRLLM_OK;
     void* base = nullptr;
     cudaError_t e = scratch_address(&base);
-    if (e != cudaSuccess) return SIRLLM_ERR_CUDA;
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress");
     cudaStream_t st = (cudaStream_t)cuda_stream;
     // status word and tickets must start at zero; the pairs are written before they are read
     e = cudaMemsetAsync(base, 0, kSsTicketsOff + (size_t)rows * 4, st);
-    if (e != cudaSuccess) return SIRLLM_ERR_CUDA;
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
     ScoreParams sp;
     sp.logits = logits;
     sp.token_ids = token_ids;
@@ -364,5 +364,5 @@ extern "C" int sirllm_score_static(const sirllm_config* cfg, const void* logits,
     sp.logits_dtype = cfg->logits_dtype;
     sp.capacity = cfg->capacity;
     e = launch_score(sp, st);
-    return e == cudaSuccess ? SIRLLM_OK : SIRLLM_ERR_CUDA;
+    return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "score");
 }
