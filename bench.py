@@ -82,7 +82,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "10"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -114,8 +114,8 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         if sm:
-            self.result = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx),
-                           "reasons": sorted(reasons), "samples": len(sm)}
+            self.result = {"sm_mhz": statistics.median(sm), "sm_min_mhz": min(sm),
+                           "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
 
 
 # --------------------------------------------------------------------------------------------
@@ -259,6 +259,14 @@ def run_ours(args, rank, world, local_rank):
         graph.replay()
         sync()
     with ClockSampler(local_rank) as clk:
+        # the sampler needs a few hundred ms of the same load to see the clocks the timed
+        # rounds run at: keep stepping (untimed) before the timed region starts
+        soak_end = time.perf_counter() + 0.3
+        while time.perf_counter() < soak_end:
+            for _ in range(8):
+                p.step()
+            torch.cuda.synchronize()
+        sync()
         t0.record()
         if graph is None:
             for _ in range(args.steps):
