@@ -6,6 +6,7 @@ arrays); bf16 / fp16 tensors are passed by their 16-bit patterns.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
 import os
 import subprocess
@@ -31,10 +32,10 @@ def build(force: bool = False) -> str:
 _lib = None
 
 
-def lib():
-    global _lib
-    if _lib is None:
-        L = ctypes.CDLL(build())
+def _bind(path: str):
+    """Load an oracle library and declare its C signatures."""
+    if True:
+        L = ctypes.CDLL(path)
         vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
         L.oracle_token_entropy.restype = ctypes.c_double
         L.oracle_token_entropy.argtypes = [vp, ctypes.c_int, i64, i32, vp]
@@ -61,8 +62,27 @@ def lib():
         L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
         L.oracle_keep_random.restype = i32
         L.oracle_keep_random.argtypes = [i32, i32, i32, i32, i32, ctypes.c_uint64, i32, i32, vp]
-        _lib = L
+    return L
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = _bind(build())
     return _lib
+
+
+@contextlib.contextmanager
+def use_library(path: str):
+    """Temporarily route every call through another build of the oracle (the tests use this
+    to check that their pins reject deliberately broken variants)."""
+    global _lib
+    saved = lib()
+    _lib = _bind(path)
+    try:
+        yield
+    finally:
+        _lib = saved
 
 
 def _ptr(x):
