@@ -40,7 +40,7 @@ WorkspaceLayout workspace_layout(const sirllm_config& c) {
     WorkspaceLayout L;
     const int64_t epv = 16 / logits_elem_bytes(c.logits_dtype);
     const int64_t nvec = c.vocab / epv;
-    const int64_t per_cta = (int64_t)kVecPerSeg * kScoreWarpsPerCta;
+    const int64_t per_cta = kScoreCtaVecs;
     L.n_part = (int32_t)((nvec + per_cta - 1) / per_cta);
     if (L.n_part < 1) L.n_part = 1;
     size_t off = 256;

@@ -27,11 +27,11 @@ struct WorkspaceLayout {
     size_t policy_ones_off;
     size_t partials_off;
     size_t total;
-    int32_t n_part;  // CTAs (groups of kScoreWarpsPerCta segments) per logits row
+    int32_t n_part;  // CTAs (kScoreCtaVecs vectors each) per logits row
 };
 
-constexpr int kVecPerSeg = 1024;  // 16-byte vectors per segment: 16 KB of logits per warp
-constexpr int kScoreWarpsPerCta = 4;
+constexpr int kScoreCtaVecs = 4096;  // 16-byte vectors of one logits row per CTA: 64 KB, shared
+                                     // by 4 warps (16 KB each) or, in small grids, 8 or 16
 constexpr int kListMax = 256;  // keys ranked directly once a radix bin holds no more
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -1,7 +1,9 @@
 // Token Entropy (Section 3.2): e = -log softmax(z)[id] as a vocabulary-streaming
-// log-sum-exp.  Every logits row is cut into segments of kVecPerSeg 16-byte vectors;
+// log-sum-exp.  Every logits row is cut into 64 KB parts, one CTA each, and every part into
+// one segment per warp;
 // one warp reduces one segment with an online (running-max) softmax sum, and the
-// kScoreWarpsPerCta warps of a CTA (consecutive segments of one row) combine their
+// the warps of a CTA (4, or 8 / 16 when the grid would otherwise leave the GPU
+// underfilled) combine their
 // (scaled max, sum) pairs through shared memory.  A row that needs several CTAs
 // (vocabularies above 32768 bf16 / 16384 fp32 elements) publishes one pair per CTA in
 // scratch; the CTA that arrives last on the row's ticket combines them.  Combination is
@@ -54,18 +56,19 @@ __device__ __forceinline__ uint32_t bf162_max(uint32_t a, uint32_t b) {
     return *reinterpret_cast<uint32_t*>(&m);
 }
 
-template <bool kBf16>
-__global__ void __launch_bounds__(kScoreWarpsPerCta * 32)
+template <bool kBf16, int kWarps>
+__global__ void __launch_bounds__(kWarps * 32)
 score_kernel(const ScoreParams p) {
+    constexpr int kVecPerSeg = kScoreCtaVecs / kWarps;
     constexpr int ES = kBf16 ? 2 : 4;
     constexpr int EPV = 16 / ES;
-    __shared__ float2 warp_pair[kScoreWarpsPerCta];
+    __shared__ float2 warp_pair[kWarps];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     grid_launch_dependents();
-    // one CTA = kScoreWarpsPerCta consecutive segments of one logits row
+    // one CTA = kWarps consecutive segments of one logits row
     const int64_t row = blockIdx.x / p.n_part;
     const int part_idx = (int)(blockIdx.x - row * p.n_part);
-    const int seg = part_idx * kScoreWarpsPerCta + wid;
+    const int seg = part_idx * kWarps + wid;
     const int s = (int)(row / p.max_new);
     const int t = (int)(row - (int64_t)s * p.max_new);
     int T = p.max_new;
@@ -164,7 +167,7 @@ score_kernel(const ScoreParams p) {
     if (wid != 0) return;
 
     // CTA combine in fp64 (fixed order): sum_v exp(z_v) over the CTA's segments = acc * 2^Mx
-    float2 q = lane < kScoreWarpsPerCta ? warp_pair[lane] : make_float2(kNegHuge, 0.f);
+    float2 q = lane < kWarps ? warp_pair[lane] : make_float2(kNegHuge, 0.f);
     float Mx = q.x;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) Mx = fmaxf(Mx, __shfl_xor_sync(0xFFFFFFFFu, Mx, o));
@@ -272,10 +275,25 @@ cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
     if (ctas == 0) return cudaSuccess;
     if (ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;
     const unsigned grid = (unsigned)ctas;
-    if (p.logits_dtype == SIRLLM_BF16)
-        score_kernel<true><<<grid, kScoreWarpsPerCta * 32, 0, st>>>(p);
-    else
-        score_kernel<false><<<grid, kScoreWarpsPerCta * 32, 0, st>>>(p);
+    // 4 warps per CTA stream 16 KB each; a grid too small to give every SM even 8 warps takes
+    // 8 or 16 warps per CTA instead (same bytes per CTA, shorter serial loop per warp).  With
+    // more warps already resident, wider CTAs measured slower.
+    int dev = 0, n_sm = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess)
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    const int64_t want_warps = (int64_t)n_sm * 8;
+    const int warps = ctas * 4 >= want_warps ? 4 : (ctas * 8 >= want_warps ? 8 : 16);
+    const bool bf16 = p.logits_dtype == SIRLLM_BF16;
+    if (warps == 4) {
+        if (bf16) score_kernel<true, 4><<<grid, 128, 0, st>>>(p);
+        else score_kernel<false, 4><<<grid, 128, 0, st>>>(p);
+    } else if (warps == 8) {
+        if (bf16) score_kernel<true, 8><<<grid, 256, 0, st>>>(p);
+        else score_kernel<false, 8><<<grid, 256, 0, st>>>(p);
+    } else {
+        if (bf16) score_kernel<true, 16><<<grid, 512, 0, st>>>(p);
+        else score_kernel<false, 16><<<grid, 512, 0, st>>>(p);
+    }
     return cudaGetLastError();
 }
 
