@@ -515,3 +515,25 @@ def test_select_randomised_shapes_and_score_patterns():
             assert torch.equal(keep[s, :n].cpu(), want), ctx
             assert torch.equal(dE[s, :n].cpu().view(torch.int32), Es[want.long()].view(torch.int32)), ctx
             assert torch.equal(dser[s, :n].cpu(), serial[s][want.long()]), ctx
+
+
+def test_step_with_optional_arguments_left_out():
+    # no tags, no keep-list / count outputs (the workspace holds them), no raw-score output,
+    # only K (V skipped), n_new = NULL meaning max_new everywhere
+    w = wl.WORKLOADS["tiny"].scaled(n_streams=2, n_layers=1, n_kv_heads=2, capacity=256, budget=96,
+                                    n_recent=16, new_tokens=70, vocab=3001)
+    a, b = DeviceState(w), DeviceState(w)
+    for r in range(3):
+        a.fill_round(r)
+        b.fill_round(r)
+        a.step()
+        B.sirllm_step(b.cfg, b.logits, b.token_ids, None, b.scores, None, b.live_len, b.decay,
+                      b.k, None, None, None, None, b.ws)
+        assert B.sirllm_status(b.ws) == 0
+        assert torch.equal(a.live_len, b.live_len)
+        n = int(a.live_len[0])
+        assert torch.equal(a.scores[:, :n].view(torch.int32), b.scores[:, :n].view(torch.int32))
+        assert torch.equal(a.k[:, :, :n], b.k[:, :, :n])
+        b.host_len = b.live_len.cpu().tolist()
+    # V was never compacted on b: its new rows still sit where they were appended
+    assert not torch.equal(a.v[:, :, :n], b.v[:, :, :n])
