@@ -537,3 +537,52 @@ def test_step_with_optional_arguments_left_out():
         b.host_len = b.live_len.cpu().tolist()
     # V was never compacted on b: its new rows still sit where they were appended
     assert not torch.equal(a.v[:, :, :n], b.v[:, :, :n])
+
+
+def test_step_host_matches_the_device_round():
+    # the same rounds once with device-resident inputs and once through sirllm_step_host
+    # (pinned host logits / ids / new K/V rows in, keep lists / lengths / raw scores out)
+    w = wl.WORKLOADS["batched64"].scaled(n_streams=3, n_layers=2, n_kv_heads=2, capacity=384,
+                                         budget=192, n_recent=32, new_tokens=80, vocab=2500)
+    a, b = DeviceState(w), DeviceState(w)
+    S, P, M, D = w.n_streams, w.planes_per_stream, w.new_tokens, w.head_dim
+    h_len = torch.zeros(S, dtype=torch.int32).pin_memory()
+    h_keep = torch.zeros(S, b.cfg.threshold, dtype=torch.int32).pin_memory()
+    h_nk = torch.zeros(S, dtype=torch.int32).pin_memory()
+    h_e = torch.zeros(S * M, dtype=torch.float32).pin_memory()
+    next_serial = 0
+    for r in range(5):
+        n_new = wl.ragged_lengths(3, S, r, M).tolist()
+        a.fill_round(r, n_new)
+        a.step()
+        # host copies of the round's inputs, generated on the CPU
+        h_logits = torch.zeros(S * M, w.vocab, dtype=w.torch_logits_dtype).pin_memory()
+        h_ids = torch.zeros(S * M, dtype=torch.int32).pin_memory()
+        h_k = torch.zeros(S, P, M, D, dtype=w.torch_kv_dtype).pin_memory()
+        h_v = torch.zeros(S, P, M, D, dtype=w.torch_kv_dtype).pin_memory()
+        for s in range(S):
+            T = n_new[s]
+            h_logits[s * M:s * M + T] = wl.make_logits(w, 0, s, r, T)
+            h_ids[s * M:s * M + T] = wl.make_token_ids(w, 0, s, r, T)
+            serials = torch.arange(b.next_serial[s], b.next_serial[s] + T)
+            h_k[s, :, :T] = wl.make_kv_rows(w, 0, "k", s, serials)
+            h_v[s, :, :T] = wl.make_kv_rows(w, 0, "v", s, serials)
+            l = int(h_len[s])
+            b.serial[s, l:l + T] = serials.to(DEV)          # tags are device state of the caller
+            b.next_serial[s] += T
+        h_n_new = torch.tensor(n_new, dtype=torch.int32).pin_memory()
+        B.sirllm_step_host(b.cfg, h_logits, h_ids, h_n_new, h_k, h_v, h_len, b.logits, b.token_ids,
+                           b.n_new, b.scores, b.serial, b.live_len, b.decay, b.k, b.v, b.keep_idx,
+                           b.n_keep, b.new_entropy, h_keep, h_nk, h_e, b.ws)
+        torch.cuda.current_stream().synchronize()
+        assert B.sirllm_status(b.ws) == 0
+        assert h_nk.tolist() == a.host_len == b.live_len.cpu().tolist()
+        h_len.copy_(h_nk)
+        for s in range(S):
+            n, T = a.host_len[s], n_new[s]
+            assert torch.equal(h_keep[s, :n], a.keep_idx[s, :n].cpu())
+            assert torch.equal(h_e[s * M:s * M + T].view(torch.int32),
+                               a.new_entropy[s * M:s * M + T].cpu().view(torch.int32))
+            assert torch.equal(a.scores[s, :n].view(torch.int32), b.scores[s, :n].view(torch.int32))
+            assert torch.equal(a.serial[s, :n], b.serial[s, :n])
+            assert torch.equal(a.k[s, :, :n], b.k[s, :, :n]) and torch.equal(a.v[s, :, :n], b.v[s, :, :n])
