@@ -62,6 +62,12 @@ def _bind(path: str):
         L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
         L.oracle_keep_random.restype = i32
         L.oracle_keep_random.argtypes = [i32, i32, i32, i32, i32, ctypes.c_uint64, i32, i32, vp]
+        L.oracle_rope_rotate_f64.restype = None
+        L.oracle_rope_rotate_f64.argtypes = [vp, i32, i32, ctypes.c_double, ctypes.c_int]
+        L.oracle_round16.restype = ctypes.c_double
+        L.oracle_round16.argtypes = [ctypes.c_double, ctypes.c_int]
+        L.oracle_rerotate_plane.restype = None
+        L.oracle_rerotate_plane.argtypes = [vp, ctypes.c_int, i32, vp, i32, ctypes.c_double, ctypes.c_int]
     return L
 
 
@@ -190,6 +196,31 @@ def keep_policy(policy: int, live_len: int, n_sink: int, n_recent: int, budget: 
     else:
         raise ValueError("unknown policy")
     return keep[:n].clone()
+
+
+ROPE_HALF, ROPE_INTERLEAVED = 0, 1
+
+
+def rope_rotate(row: torch.Tensor, delta: int, base: float, layout: int) -> torch.Tensor:
+    """A float64 row turned by ``delta`` positions of rotary embedding (new tensor)."""
+    out = row.to(torch.float64).contiguous().clone()
+    lib().oracle_rope_rotate_f64(_ptr(out), out.numel(), int(delta), float(base), int(layout))
+    return out
+
+
+def round16(v: float, bf16: bool) -> float:
+    return lib().oracle_round16(float(v), int(bf16))
+
+
+def rerotate_plane(plane: torch.Tensor, keep: torch.Tensor, base: float, layout: int) -> torch.Tensor:
+    """Copy of a K plane ``[slots, d]`` (bf16/fp16) whose rows j < len(keep) are turned by
+    ``j - keep[j]`` positions."""
+    assert plane.dtype in (torch.bfloat16, torch.float16) and plane.dim() == 2
+    out = plane.contiguous().clone()
+    keep = keep.to(torch.int32).contiguous()
+    lib().oracle_rerotate_plane(_ptr(out), int(plane.dtype == torch.bfloat16), out.shape[1], _ptr(keep),
+                                keep.numel(), float(base), int(layout))
+    return out
 
 
 class Stream:

@@ -368,3 +368,110 @@ int32_t oracle_keep_random(int32_t l, int32_t n_sink, int32_t n_recent, int32_t 
     qsort(keep, (size_t)n, sizeof(int32_t), by_int_asc);
     return n;
 }
+
+/* ---- re-indexing of positions for caches that hold keys AFTER rotary embedding ----------
+ * Section 3.3 (the paragraph on positions): a token's position is its place inside the cache,
+ * not in the text; after an eviction the kept tokens take positions 0..n-1 in slot order.  A
+ * model that stores keys already rotated for the position they were written at therefore has
+ * to turn the key that moved from slot keep[j] to slot j by the angle of (j - keep[j])
+ * positions.  Rotary embedding (Su et al., RoFormer): pair i of a row, i < d/2, is the complex
+ * number x + iy turned by the angle  position * theta_i,  theta_i = base^(-2i/d);
+ * layout 0 pairs (row[i], row[i + d/2]), layout 1 pairs (row[2i], row[2i+1]). */
+#define ORACLE_ROPE_HALF 0
+#define ORACLE_ROPE_INTERLEAVED 1
+
+void oracle_rope_rotate_f64(double *row, int32_t d, int32_t delta, double base, int layout)
+{
+    int32_t hp = d / 2;
+    for (int32_t i = 0; i < hp; ++i) {
+        double theta = pow(base, -2.0 * (double)i / (double)d);
+        double ang = (double)delta * theta, c = cos(ang), s = sin(ang);
+        double *px = layout == ORACLE_ROPE_HALF ? &row[i] : &row[2 * i];
+        double *py = layout == ORACLE_ROPE_HALF ? &row[i + hp] : &row[2 * i + 1];
+        double x = *px, y = *py;
+        *px = x * c - y * s;
+        *py = x * s + y * c;
+    }
+}
+
+/* Round a double to the nearest value with `p` significant bits and minimum exponent
+ * `emin` (ties to even; needs the default rounding mode), i.e. to bf16 (p = 8, emin = -126)
+ * or fp16 (p = 11, emin = -14) without passing through fp32. */
+static double round_to_format(double v, int p, int emin)
+{
+    if (v == 0.0 || isnan(v) || isinf(v))
+        return v;
+    int e;
+    double m = frexp(v, &e); /* v = m * 2^e, 0.5 <= |m| < 1: the leading bit has weight 2^(e-1) */
+    int keep = p;
+    if (e - 1 < emin)
+        keep = p - (emin - (e - 1)); /* subnormal: fewer bits */
+    if (keep <= 0)
+        return ldexp(nearbyint(ldexp(v, -(emin - p + 1))), emin - p + 1);
+    return ldexp(nearbyint(ldexp(m, keep)), e - keep);
+}
+
+static double from_bits16(uint16_t h, int dtype_is_bf16)
+{
+    if (dtype_is_bf16) {
+        uint32_t b = (uint32_t)h << 16;
+        float f;
+        memcpy(&f, &b, sizeof f);
+        return (double)f;
+    }
+    int sign = h >> 15, ex = (h >> 10) & 31, fr = h & 1023;
+    double v = ex == 0 ? ldexp((double)fr, -24) : ex == 31 ? (fr ? NAN : INFINITY)
+                                                            : ldexp((double)(fr | 1024), ex - 25);
+    return sign ? -v : v;
+}
+
+static uint16_t to_bits16(double v, int dtype_is_bf16)
+{
+    double r = dtype_is_bf16 ? round_to_format(v, 8, -126) : round_to_format(v, 11, -14);
+    if (dtype_is_bf16) {
+        float f = (float)r; /* exact: r has 8 significant bits */
+        if (isinf(f) && !isinf(v))
+            f = copysignf(INFINITY, f);
+        uint32_t b;
+        memcpy(&b, &f, sizeof b);
+        return (uint16_t)(b >> 16);
+    }
+    uint16_t sign = signbit(r) ? 0x8000u : 0;
+    double a = fabs(r);
+    if (isnan(a))
+        return sign | 0x7E00u;
+    if (a >= 65520.0)
+        return sign | 0x7C00u;
+    if (a == 0.0)
+        return sign;
+    int e;
+    double m = frexp(a, &e); /* a = m 2^e */
+    if (e - 1 < -14)
+        return sign | (uint16_t)ldexp(a, 24); /* subnormal: a / 2^-24, an integer < 1024 */
+    return sign | (uint16_t)(((e - 1 + 15) << 10) | ((int)ldexp(m, 11) & 1023));
+}
+
+double oracle_round16(double v, int dtype_is_bf16)
+{
+    return from_bits16(to_bits16(v, dtype_is_bf16), dtype_is_bf16);
+}
+
+/* Re-rotate the live rows of one K plane in place: row j by (j - keep[j]) positions, computed
+ * in double and rounded once to the storage type.  plane: [slots][d] 16-bit elements. */
+void oracle_rerotate_plane(void *plane, int dtype_is_bf16, int32_t d, const int32_t *keep,
+                           int32_t n_keep, double base, int layout)
+{
+    double *row = malloc(sizeof(double) * (size_t)d);
+    for (int32_t j = 0; j < n_keep; ++j) {
+        int32_t delta = j - keep[j];
+        if (delta == 0)
+            continue;
+        uint16_t *h = (uint16_t *)plane + (size_t)j * (size_t)d;
+        for (int32_t c = 0; c < d; ++c)
+            row[c] = from_bits16(h[c], dtype_is_bf16);
+        oracle_rope_rotate_f64(row, d, delta, base, layout);
+        for (int32_t c = 0; c < d; ++c)
+            h[c] = to_bits16(row[c], dtype_is_bf16);
+    }
+    free(row);
+}

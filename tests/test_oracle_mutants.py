@@ -9,6 +9,7 @@ import pytest
 import oracle
 import test_oracle_pairs as t_pairs
 import test_oracle_policies as t_pol
+import test_oracle_rope as t_rope
 import test_oracle_score as t_score
 import test_oracle_select as t_sel
 import test_oracle_step as t_step
@@ -59,6 +60,14 @@ MUTANTS = {
     "random policy: round not part of the counter":
         ("uint32_t ctr[4] = {(uint32_t)i, (uint32_t)round, (uint32_t)stream, 0u}, out[4];",
          "uint32_t ctr[4] = {(uint32_t)i, 0u, (uint32_t)stream, 0u}, out[4];"),
+    "rope: rotation the wrong way round":
+        ("        *px = x * c - y * s;\n        *py = x * s + y * c;", "        *px = x * c + y * s;\n        *py = -x * s + y * c;"),
+    "rope: frequencies base^(-i/d)":
+        ("double theta = pow(base, -2.0 * (double)i / (double)d);", "double theta = pow(base, -1.0 * (double)i / (double)d);"),
+    "rope: turned by the new position instead of the shift":
+        ("        int32_t delta = j - keep[j];", "        int32_t delta = j;"),
+    "rope: storage rounding truncates":
+        ("return ldexp(nearbyint(ldexp(m, keep)), e - keep);", "return ldexp(trunc(ldexp(m, keep)), e - keep);"),
     "philox: nine rounds":
         ("for (int r = 0; r < 10; ++r) {", "for (int r = 0; r < 9; ++r) {"),
 }
@@ -67,7 +76,7 @@ MUTANTS = {
 def _pins():
     """The regular pins, as plain callables."""
     calls = []
-    for mod in (t_score, t_sel, t_step, t_pairs, t_pol):
+    for mod in (t_score, t_sel, t_step, t_pairs, t_pol, t_rope):
         for name in sorted(dir(mod)):
             fn = getattr(mod, name)
             if not name.startswith("test_") or not callable(fn):
