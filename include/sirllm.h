@@ -62,6 +62,10 @@ extern "C" {
 #define SIRLLM_POLICY_RANDOM 2
 #define SIRLLM_POLICY_INTERVAL 3
 
+/* pairing of a key row's elements under rotary embedding, for sirllm_rerotate_keys */
+#define SIRLLM_ROPE_HALF 0        /* pair i = (row[i], row[i + head_dim/2]) */
+#define SIRLLM_ROPE_INTERLEAVED 1 /* pair i = (row[2i], row[2i+1]) */
+
 /* Largest `capacity` the selection kernel supports (the scores of one stream are
  * held in one SM's shared memory). */
 #define SIRLLM_MAX_CAPACITY 49152
@@ -215,6 +219,23 @@ int sirllm_keep_policy(const sirllm_config *cfg, int32_t policy, const int32_t *
 int sirllm_compact_kv(const sirllm_config *cfg, const void *k_src, const void *v_src, void *k_dst,
                       void *v_dst, const int32_t *keep_idx, const int32_t *n_keep, void *ws,
                       void *cuda_stream);
+
+/*
+ * Positions inside the cache for models that store keys AFTER rotary position embedding
+ * (Section 3.3: positions are assigned by place in the cache, not in the text; the printed
+ * example gives tokens [0,1,2,3,5,7,11,12] the positions [0..7]).  Call after K has been
+ * compacted with the same keep lists: the key now in slot j was written for position
+ * keep_idx[s][j]; it is turned by (j - keep_idx[s][j]) positions, pair i of the row by the
+ * angle shift * rope_base^(-2i/head_dim), so that it becomes the key of a token at position
+ * j.  Rows that did not move are not touched.  Angles are evaluated in fp64, the rotation in
+ * fp32, and each element is rounded once to the K dtype.  (A model that caches keys before
+ * the rotary embedding needs no such call: slot order already is the position.)
+ *   k         the K cache of sirllm_compact_kv, updated in place; head_dim % 16 == 0
+ *   rope_base the base of the frequencies (10000, 500000, ...); layout: SIRLLM_ROPE_*
+ */
+int sirllm_rerotate_keys(const sirllm_config *cfg, void *k, const int32_t *keep_idx,
+                         const int32_t *n_keep, double rope_base, int32_t layout,
+                         void *cuda_stream);
 
 /*
  * One whole round (Algorithm 1's loop body): score the n_new[s] new tokens, append

@@ -21,9 +21,10 @@ OK, ERR_NULL, ERR_BAD_CONFIG, ERR_ALIGN, ERR_CUDA, ERR_TOO_LARGE = 0, -1, -2, -3
 STATUS_TOKEN_RANGE, STATUS_OVERFLOW, STATUS_TIMEOUT, STATUS_BAD_KEEP = 1, 2, 4, 8
 MAX_CAPACITY = 49152
 POLICY_STREAM, POLICY_RANDOM, POLICY_INTERVAL = 1, 2, 3
+ROPE_HALF, ROPE_INTERLEAVED = 0, 1
 
 EXPORTS = ["sirllm_workspace_bytes", "sirllm_workspace_init", "sirllm_score", "sirllm_score_static",
-           "sirllm_score_pairs", "sirllm_step_pairs", "sirllm_decay_select", "sirllm_keep_policy",
+           "sirllm_score_pairs", "sirllm_step_pairs", "sirllm_decay_select", "sirllm_keep_policy", "sirllm_rerotate_keys",
            "sirllm_compact_kv", "sirllm_step", "sirllm_step_phases", "sirllm_step_host",
            "sirllm_status", "sirllm_strerror",
            "sirllm_last_cuda_error"]
@@ -97,6 +98,8 @@ def lib():
         L.sirllm_decay_select.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, i32, vp, vp]
         L.sirllm_keep_policy.restype = ctypes.c_int
         L.sirllm_keep_policy.argtypes = [cfgp, i32, vp, ctypes.c_uint64, i32, i32, vp, vp, vp, vp]
+        L.sirllm_rerotate_keys.restype = ctypes.c_int
+        L.sirllm_rerotate_keys.argtypes = [cfgp, vp, vp, vp, ctypes.c_double, i32, vp]
         L.sirllm_compact_kv.restype = ctypes.c_int
         L.sirllm_compact_kv.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.sirllm_step.restype = ctypes.c_int
@@ -248,6 +251,14 @@ def sirllm_keep_policy(cfg: Config, policy: int, live_len, seed: int, rnd: int, 
 
 
 _KV = (torch.bfloat16, torch.float16)
+
+
+def sirllm_rerotate_keys(cfg: Config, k, keep_idx, n_keep, rope_base: float, layout: int) -> None:
+    """Turns the moved rows of a compacted post-rotary K cache to their new positions."""
+    _check(lib().sirllm_rerotate_keys(ctypes.byref(cfg), _dev(k, _KV, "k"),
+                                      _dev(keep_idx, torch.int32, "keep_idx"),
+                                      _dev(n_keep, torch.int32, "n_keep"), float(rope_base),
+                                      int(layout), _stream()))
 
 
 def sirllm_compact_kv(cfg: Config, k_src, v_src, k_dst, v_dst, keep_idx, n_keep, ws) -> None:

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsirllm.so")
-SOURCES = ["api.cu", "score.cu", "select.cu", "compact.cu", "policy.cu"]
+SOURCES = ["api.cu", "score.cu", "select.cu", "compact.cu", "policy.cu", "rope.cu"]
 
 
 def _stale() -> bool:

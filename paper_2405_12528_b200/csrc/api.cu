@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in sirllm.h: argument checks, workspace layout and
 // the launch sequences.  No device memory is allocated here.
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 
@@ -464,6 +465,31 @@ int sirllm_keep_policy(const sirllm_config* cfg, int32_t policy, const int32_t* 
                        int32_t* n_keep, void* ws, void* cuda_stream) {
     return keep_policy_impl(cfg, policy, live_len, seed, round, stream_base, keep_idx, n_keep,
                                    ws, cuda_stream);
+}
+
+int sirllm_rerotate_keys(const sirllm_config* cfg, void* k, const int32_t* keep_idx,
+                         const int32_t* n_keep, double rope_base, int32_t layout, void* cuda_stream) {
+    int rc = validate_config(cfg);
+    if (rc != SIRLLM_OK) return rc;
+    if (!k || !keep_idx || !n_keep) return SIRLLM_ERR_NULL;
+    if (misaligned(k, 16)) return SIRLLM_ERR_ALIGN;
+    if (cfg->head_dim % 16 != 0 || !(rope_base > 0.0) || !std::isfinite(rope_base) ||
+        (layout != SIRLLM_ROPE_HALF && layout != SIRLLM_ROPE_INTERLEAVED))
+        return SIRLLM_ERR_BAD_CONFIG;
+    RopeParams p;
+    p.k = (char*)k;
+    p.keep_idx = keep_idx;
+    p.n_keep = n_keep;
+    p.log2_base = std::log2(rope_base);
+    p.capacity = cfg->capacity;
+    p.keep_stride = cfg->threshold;
+    p.planes_per_stream = cfg->n_layers * cfg->n_kv_heads;
+    p.head_dim = cfg->head_dim;
+    p.layout = layout;
+    p.planes_per_group = p.planes_per_stream;
+    cudaError_t e = launch_rerotate(p, cfg->n_streams, cfg->kv_dtype == SIRLLM_BF16,
+                                    (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "rerotate");
 }
 
 int sirllm_status(void* ws, void* cuda_stream, int32_t* status_out, int32_t clear) {

@@ -95,6 +95,14 @@ struct PolicyParams {
     int32_t policy, round, stream_base, capacity, budget, n_sink;
 };
 
+struct RopeParams {
+    char* k;
+    const int32_t* keep_idx;
+    const int32_t* n_keep;
+    double log2_base;
+    int32_t capacity, keep_stride, planes_per_stream, head_dim, layout, planes_per_group;
+};
+
 struct CompactParams {
     const char* src[2];  // K, V (nullable)
     char* dst[2];
@@ -117,6 +125,7 @@ cudaError_t launch_score_pairs(const PairScoreParams& p, cudaStream_t st);
 // results (grid_dependency_wait) before it reads them.
 cudaError_t launch_select(const SelectParams& p, int n_streams, cudaStream_t st, bool overlap);
 cudaError_t launch_policy_ranks(const PolicyParams& p, int n_streams, cudaStream_t st);
+cudaError_t launch_rerotate(const RopeParams& p, int n_streams, bool bf16, cudaStream_t st);
 cudaError_t launch_compact_plan(const CompactParams& p, int n_streams, int32_t* first_moved,
                                 cudaStream_t st);
 cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap);

@@ -1,0 +1,125 @@
+// Positions inside the cache for keys stored AFTER rotary embedding (Section 3.3, the
+// paragraph on positions): once compaction has moved the key of slot keep[j] to slot j, the
+// key is turned by the angle of (j - keep[j]) positions so that it is again the key of a token
+// at position j.  Rotary embedding (Su et al., RoFormer): pair i < d/2 of a row is a complex
+// number turned by  position * theta_i,  theta_i = base^(-2i/d).
+//
+// Bound by HBM traffic on the moved rows of the K planes (read once, written once).  The
+// angles depend on (stream, slot, pair) only, so a thread computes its eight (cos, sin) once -
+// in fp64, the shift can be thousands of positions - and reuses them for every K plane of its
+// group; per plane it moves two 16-byte vectors, rotates in fp32 and rounds once to bf16/fp16.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+
+namespace sirllm {
+
+namespace {
+
+constexpr int kRopeThreads = 128;
+
+template <bool kBf16>
+__device__ __forceinline__ float load16(uint32_t word, int hi) {
+    const uint16_t h = hi ? (uint16_t)(word >> 16) : (uint16_t)(word & 0xFFFFu);
+    if (kBf16) return __uint_as_float((uint32_t)h << 16);
+    return __half2float(__ushort_as_half(h));
+}
+template <bool kBf16>
+__device__ __forceinline__ uint32_t pack16(float lo, float hi) {
+    if (kBf16) {
+        return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) |
+               ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+    }
+    return (uint32_t)__half_as_ushort(__float2half_rn(lo)) |
+           ((uint32_t)__half_as_ushort(__float2half_rn(hi)) << 16);
+}
+
+template <bool kBf16>
+__global__ void __launch_bounds__(kRopeThreads) rerotate_kernel(const RopeParams p) {
+    const int units = p.head_dim / 16;  // threads per row: 8 pairs (two 16-byte vectors) each
+    const int rows_per_block = kRopeThreads / units;
+    const int r = threadIdx.x / units, u = threadIdx.x - r * units;
+    if (r >= rows_per_block) return;
+    const int s = blockIdx.y;
+    const int j = blockIdx.x * rows_per_block + r;
+    if (j >= min(p.n_keep[s], p.keep_stride)) return;
+    const int delta = j - p.keep_idx[(size_t)s * p.keep_stride + j];
+    if (delta == 0) return;  // the row did not move
+
+    float cs[8], sn[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const int i = 8 * u + q;
+        const double theta = exp2(-(double)(2 * i) / (double)p.head_dim * p.log2_base);
+        double sv, cv;
+        sincos((double)delta * theta, &sv, &cv);
+        cs[q] = (float)cv;
+        sn[q] = (float)sv;
+    }
+    const size_t row_bytes = (size_t)p.head_dim * 2;
+    const int pl0 = blockIdx.z * p.planes_per_group;
+    const int pl1 = min(p.planes_per_stream, pl0 + p.planes_per_group);
+    for (int pl = pl0; pl < pl1; ++pl) {
+        char* row = p.k + (((size_t)s * p.planes_per_stream + pl) * p.capacity + j) * row_bytes;
+        uint4* pa = reinterpret_cast<uint4*>(row + (p.layout == SIRLLM_ROPE_HALF ? 16 * u : 32 * u));
+        uint4* pb = reinterpret_cast<uint4*>(
+            row + (p.layout == SIRLLM_ROPE_HALF ? (size_t)p.head_dim + 16 * u : 32 * u + 16));
+        const uint4 a = *pa, b = *pb;
+        const uint32_t wa[4] = {a.x, a.y, a.z, a.w}, wb[4] = {b.x, b.y, b.z, b.w};
+        uint32_t oa[4], ob[4];
+        if (p.layout == SIRLLM_ROPE_HALF) {  // a holds x of pairs 8u..8u+7, b holds their y
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float x[2], y[2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float xv = load16<kBf16>(wa[q], h), yv = load16<kBf16>(wb[q], h);
+                    x[h] = fmaf(xv, cs[2 * q + h], -(yv * sn[2 * q + h]));
+                    y[h] = fmaf(xv, sn[2 * q + h], yv * cs[2 * q + h]);
+                }
+                oa[q] = pack16<kBf16>(x[0], x[1]);
+                ob[q] = pack16<kBf16>(y[0], y[1]);
+            }
+        } else {  // every 32-bit word is one pair (x, y): a = pairs 8u..8u+3, b = 8u+4..8u+7
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float xv = load16<kBf16>(wa[q], 0), yv = load16<kBf16>(wa[q], 1);
+                oa[q] = pack16<kBf16>(fmaf(xv, cs[q], -(yv * sn[q])), fmaf(xv, sn[q], yv * cs[q]));
+                xv = load16<kBf16>(wb[q], 0);
+                yv = load16<kBf16>(wb[q], 1);
+                ob[q] = pack16<kBf16>(fmaf(xv, cs[4 + q], -(yv * sn[4 + q])),
+                                      fmaf(xv, sn[4 + q], yv * cs[4 + q]));
+            }
+        }
+        *pa = make_uint4(oa[0], oa[1], oa[2], oa[3]);
+        *pb = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_rerotate(const RopeParams& p, int n_streams, bool bf16, cudaStream_t st) {
+    const int units = p.head_dim / 16;
+    const int rows_per_block = kRopeThreads / units;
+    const unsigned gx = (unsigned)((p.keep_stride + rows_per_block - 1) / rows_per_block);
+    int dev = 0, n_sm = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess)
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    // enough blocks to fill the GPU a few times over; each block reuses its angles over a group
+    // of planes
+    int64_t groups = ((int64_t)8 * n_sm + (int64_t)gx * n_streams - 1) / ((int64_t)gx * n_streams);
+    if (groups < 1) groups = 1;
+    if (groups > p.planes_per_stream) groups = p.planes_per_stream;
+    RopeParams q = p;
+    q.planes_per_group = (int32_t)((p.planes_per_stream + groups - 1) / groups);
+    const unsigned gz = (unsigned)((p.planes_per_stream + q.planes_per_group - 1) / q.planes_per_group);
+    dim3 grid(gx, (unsigned)n_streams, gz);
+    if (bf16)
+        rerotate_kernel<true><<<grid, kRopeThreads, 0, st>>>(q);
+    else
+        rerotate_kernel<false><<<grid, kRopeThreads, 0, st>>>(q);
+    return cudaGetLastError();
+}
+
+}  // namespace sirllm

@@ -586,3 +586,65 @@ def test_step_host_matches_the_device_round():
             assert torch.equal(a.scores[s, :n].view(torch.int32), b.scores[s, :n].view(torch.int32))
             assert torch.equal(a.serial[s, :n], b.serial[s, :n])
             assert torch.equal(a.k[s, :, :n], b.k[s, :, :n]) and torch.equal(a.v[s, :, :n], b.v[s, :, :n])
+
+
+# ------------------------------------------------------------------------------- rotary re-indexing
+
+def _ordered16(t):
+    b = t.view(torch.int16).to(torch.int32)
+    return torch.where(b < 0, -(b & 0x7FFF), b)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("layout", [B.ROPE_HALF, B.ROPE_INTERLEAVED])
+def test_rerotate_keys_matches_oracle(dtype, layout):
+    # the oracle rotates in fp64 and rounds once; the kernel takes fp64 angles, rotates in fp32 and
+    # rounds once: results agree bit for bit except where fp32 lands on the other side of a
+    # rounding boundary (at most one unit in the last place, on a tiny share of the elements)
+    S, P, cap, D, thr = 2, 3, 700, 128, 400
+    cfg = B.make_config(S, P, 1, D, cap, thr, 0, 0, 0, 16, torch.float32, dtype)
+    g = torch.Generator().manual_seed(layout + 7)
+    k = (torch.randn(S, P, cap, D, generator=g) * 2).to(dtype)
+    n_list = [400, 123]
+    keep = torch.full((S, thr), -1, dtype=torch.int32)
+    for s, n in enumerate(n_list):
+        picked = torch.sort(torch.randperm(cap - 20, generator=g)[:n - 20]).values + 20
+        keep[s, :n] = torch.cat([torch.arange(20), picked]).to(torch.int32)    # 20 rows stay put
+    dk = k.to(DEV)
+    B.sirllm_rerotate_keys(cfg, dk, keep.to(DEV), torch.tensor(n_list, dtype=torch.int32, device=DEV),
+                           10000.0, layout)
+    got = dk.cpu()
+    n_elems = n_off = 0
+    for s, n in enumerate(n_list):
+        for p in range(P):
+            want = oracle.rerotate_plane(k[s, p], keep[s, :n], 10000.0, layout)
+            assert torch.equal(got[s, p, n:], k[s, p, n:])                     # beyond the live rows
+            assert torch.equal(got[s, p, :20], k[s, p, :20])                   # rows that did not move
+            d = (_ordered16(got[s, p, :n]) - _ordered16(want[:n])).abs()
+            assert int(d.max()) <= 1
+            n_off += int((d != 0).sum())
+            n_elems += d.numel()
+            assert not torch.equal(got[s, p, 20:n], k[s, p, 20:n])
+    assert n_off <= 1e-3 * n_elems, (n_off, n_elems)
+
+
+def test_rerotate_after_compaction_equals_keys_written_at_their_new_positions():
+    # keys are stored rotated for the slot they were written to; after eviction + re-indexing
+    # every kept key must equal (to storage rounding) the same token's key rotated for its new slot
+    S, P, cap, D, n = 1, 2, 300, 64, 180
+    cfg = B.make_config(S, P, 1, D, cap, n, 0, 0, 0, 16, torch.float32, torch.float16)
+    ws = B.new_workspace(cfg)
+    g = torch.Generator().manual_seed(11)
+    raw = torch.randn(P, cap, D, generator=g, dtype=torch.float64)              # keys before rotation
+    stored = torch.stack([torch.stack([oracle.rope_rotate(raw[p, j], j, 10000.0, B.ROPE_HALF)
+                                       for j in range(cap)]) for p in range(P)]).to(torch.float16)
+    keep = torch.sort(torch.randperm(cap, generator=g)[:n]).values.to(torch.int32).view(1, n)
+    dk = stored.view(1, P, cap, D).to(DEV)
+    nk = torch.tensor([n], dtype=torch.int32, device=DEV)
+    B.sirllm_compact_kv(cfg, dk, None, dk, None, keep.to(DEV), nk, ws)
+    B.sirllm_rerotate_keys(cfg, dk, keep.to(DEV), nk, 10000.0, B.ROPE_HALF)
+    got = dk.cpu()[0].double()
+    for p in range(P):
+        for j in range(0, n, 7):
+            fresh = oracle.rope_rotate(raw[p, int(keep[0, j])], j, 10000.0, B.ROPE_HALF)
+            assert torch.allclose(got[p, j], fresh, rtol=0, atol=8e-3)          # two fp16 roundings
