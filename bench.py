@@ -371,6 +371,14 @@ def run_extras(p: Pass, args):
 
     out = {"pairs_tile": tile,
            "step_pairs_ms": round(_time_rounds(pairs_round, args.steps), 4)}
+    if w.head_dim % 16 == 0:
+        p.step()                                   # an entropy-selected keep list
+        # rotary re-indexing of the K rows the last compaction moved (keep lists of that round)
+        ms = _time_rounds(lambda: B.sirllm_rerotate_keys(cfg, p.k, p.keep_idx, p.n_keep, 500000.0,
+                                                         B.ROPE_HALF), args.steps)
+        moved = p.moved_rows()
+        out["rerotate_ms"] = round(ms, 4)
+        out["rerotate_gbs"] = round(2 * moved * w.row_bytes * w.planes_per_stream / (ms * 1e-3) / 1e9, 1)
     full = torch.full_like(p.live_len, w.budget + w.new_tokens)
     for name, pol in (("stream", B.POLICY_STREAM), ("random", B.POLICY_RANDOM), ("interval", B.POLICY_INTERVAL)):
         def policy_round():

@@ -600,7 +600,8 @@ def _ordered16(t):
 def test_rerotate_keys_matches_oracle(dtype, layout):
     # the oracle rotates in fp64 and rounds once; the kernel takes fp64 angles, rotates in fp32 and
     # rounds once: results agree bit for bit except where fp32 lands on the other side of a
-    # rounding boundary (at most one unit in the last place, on a tiny share of the elements)
+    # rounding boundary - one unit in the last place, or, where x*cos - y*sin cancels to a result
+    # far smaller than its inputs, the fp32 error of the products (2^-22 of the row's magnitude)
     S, P, cap, D, thr = 2, 3, 700, 128, 400
     cfg = B.make_config(S, P, 1, D, cap, thr, 0, 0, 0, 16, torch.float32, dtype)
     g = torch.Generator().manual_seed(layout + 7)
@@ -621,7 +622,9 @@ def test_rerotate_keys_matches_oracle(dtype, layout):
             assert torch.equal(got[s, p, n:], k[s, p, n:])                     # beyond the live rows
             assert torch.equal(got[s, p, :20], k[s, p, :20])                   # rows that did not move
             d = (_ordered16(got[s, p, :n]) - _ordered16(want[:n])).abs()
-            assert int(d.max()) <= 1
+            err = (got[s, p, :n].double() - want[:n].double()).abs()
+            scale = k[s, p, :n].double().abs().amax(dim=1, keepdim=True)
+            assert bool(((d <= 1) | (err <= scale * 2.0 ** -22)).all())
             n_off += int((d != 0).sum())
             n_elems += d.numel()
             assert not torch.equal(got[s, p, 20:n], k[s, p, 20:n])
