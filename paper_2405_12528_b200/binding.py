@@ -79,7 +79,13 @@ def lib():
     global _lib
     if _lib is None:
         if not os.path.exists(_LIB_PATH):
-            raise SirllmError(ERR_CUDA, f"{_LIB_PATH} not built; run paper_2405_12528_b200/build.py")
+            # a source checkout: compile once with nvcc; without a compiler this fails loudly
+            try:
+                from . import build as _build
+                _build.build()
+            except Exception as exc:
+                raise SirllmError(ERR_CUDA, f"{_LIB_PATH} is not built and could not be compiled "
+                                            f"({exc}); run paper_2405_12528_b200/build.py") from exc
         L = ctypes.CDLL(_LIB_PATH)
         vp, i32, cfgp = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(Config)
         L.sirllm_workspace_bytes.restype = ctypes.c_size_t

@@ -29,3 +29,12 @@ def pytest_collection_modifyitems(config, items):
 @pytest.fixture(scope="session")
 def golden_dir():
     return os.path.join(ROOT, "tests", "golden")
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _native_libraries():
+    """Build the CUDA library and the C oracle once per session if they are missing or stale."""
+    from paper_2405_12528_b200 import build as builder
+    import oracle
+    builder.build()
+    oracle.build()
