@@ -651,3 +651,13 @@ def test_rerotate_after_compaction_equals_keys_written_at_their_new_positions():
         for j in range(0, n, 7):
             fresh = oracle.rope_rotate(raw[p, int(keep[0, j])], j, 10000.0, B.ROPE_HALF)
             assert torch.allclose(got[p, j], fresh, rtol=0, atol=8e-3)          # two fp16 roundings
+
+
+def test_compact_in_place_with_planes_cut_into_many_chained_segments():
+    # few planes and long keep lists: every plane is cut into the maximum number of segments
+    # that different SMs take, so correctness rests on the progress-word chain; large and small
+    # displacements, a stream that moves nothing and one that moves a single row
+    _compact_case(4, 1, 20000, 128, [15000, 19999, 20000, 2], True, 21)
+    _compact_case(1, 2, 49152, 64, [30000], True, 22)
+    # out of place with the same cut (no chain needed, all rows copied)
+    _compact_case(2, 1, 20000, 128, [15000, 777], False, 23)
