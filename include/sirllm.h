@@ -295,6 +295,14 @@ int sirllm_step_host(const sirllm_config *cfg, const void *h_logits, const int32
                      float *new_entropy, int32_t *h_keep_idx, int32_t *h_n_keep,
                      float *h_new_entropy, void *ws, void *cuda_stream);
 
+/* Exercises the failure path of the library's device-side waits without a failure: one
+ * thread polls a progress word of `ws` that nothing ever sets, `polls` times (<= 2^20, a few
+ * hundred milliseconds at most), gives up exactly as the KV gather would and raises
+ * SIRLLM_STATUS_TIMEOUT; the GPU and the context stay usable.  Read the result with
+ * sirllm_status().  No counterpart in the paper. */
+int sirllm_selftest_bounded_wait(const sirllm_config *cfg, void *ws, uint32_t polls,
+                                 void *cuda_stream);
+
 /* Waits for the stream, copies the status word to *status_out (host) and, if
  * `clear` != 0, resets it.  No counterpart in the paper. */
 int sirllm_status(void *ws, void *cuda_stream, int32_t *status_out, int32_t clear);

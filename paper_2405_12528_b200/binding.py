@@ -26,7 +26,7 @@ ROPE_HALF, ROPE_INTERLEAVED = 0, 1
 EXPORTS = ["sirllm_workspace_bytes", "sirllm_workspace_init", "sirllm_score", "sirllm_score_static",
            "sirllm_score_pairs", "sirllm_step_pairs", "sirllm_decay_select", "sirllm_keep_policy", "sirllm_rerotate_keys",
            "sirllm_compact_kv", "sirllm_step", "sirllm_step_phases", "sirllm_step_host",
-           "sirllm_status", "sirllm_strerror",
+           "sirllm_selftest_bounded_wait", "sirllm_status", "sirllm_strerror",
            "sirllm_last_cuda_error"]
 
 _DTYPE_CODE = {torch.float32: F32, torch.bfloat16: BF16, torch.float16: F16}
@@ -114,6 +114,8 @@ def lib():
         L.sirllm_step_phases.argtypes = [cfgp] + [vp] * 14 + [ctypes.POINTER(vp)]
         L.sirllm_step_host.restype = ctypes.c_int
         L.sirllm_step_host.argtypes = [cfgp] + [vp] * 23
+        L.sirllm_selftest_bounded_wait.restype = ctypes.c_int
+        L.sirllm_selftest_bounded_wait.argtypes = [cfgp, vp, ctypes.c_uint32, vp]
         L.sirllm_status.restype = ctypes.c_int
         L.sirllm_status.argtypes = [vp, vp, ctypes.POINTER(i32), i32]
         L.sirllm_strerror.restype = ctypes.c_char_p
@@ -342,6 +344,12 @@ def sirllm_step_host(cfg: Config, h_logits, h_token_ids, h_n_new, h_new_k, h_new
         _dev(new_entropy, torch.float32, "new_entropy"), _host(h_keep_idx, torch.int32, "h_keep_idx"),
         _host(h_n_keep, torch.int32, "h_n_keep"), _host(h_new_entropy, torch.float32, "h_new_entropy"),
         _dev(ws, torch.uint8, "ws"), _stream()))
+
+
+def sirllm_selftest_bounded_wait(cfg: Config, ws: torch.Tensor, polls: int = 2000) -> None:
+    """Lets one device-side bounded wait run out on purpose (raises STATUS_TIMEOUT in ``ws``)."""
+    _check(lib().sirllm_selftest_bounded_wait(ctypes.byref(cfg), _dev(ws, torch.uint8, "ws"),
+                                              int(polls), _stream()))
 
 
 def sirllm_status(ws: torch.Tensor, clear: bool = False) -> int:

@@ -492,6 +492,19 @@ int sirllm_rerotate_keys(const sirllm_config* cfg, void* k, const int32_t* keep_
     return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "rerotate");
 }
 
+int sirllm_selftest_bounded_wait(const sirllm_config* cfg, void* ws, uint32_t polls,
+                                 void* cuda_stream) {
+    int rc = validate_config(cfg);
+    if (rc != SIRLLM_OK) return rc;
+    if (!ws) return SIRLLM_ERR_NULL;
+    if (misaligned(ws, 256)) return SIRLLM_ERR_ALIGN;
+    if (polls > (1u << 20)) return SIRLLM_ERR_BAD_CONFIG;  // keep the self-test short
+    const WorkspaceLayout L = workspace_layout(*cfg);
+    cudaError_t e = launch_bounded_wait_selftest((int32_t*)((char*)ws + L.plane_flags_off), polls,
+                                                 (int32_t*)ws, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "bounded_wait_selftest");
+}
+
 int sirllm_status(void* ws, void* cuda_stream, int32_t* status_out, int32_t clear) {
     if (!ws || !status_out) return SIRLLM_ERR_NULL;
     cudaStream_t st = (cudaStream_t)cuda_stream;

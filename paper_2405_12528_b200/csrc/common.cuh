@@ -129,6 +129,8 @@ cudaError_t launch_rerotate(const RopeParams& p, int n_streams, bool bf16, cudaS
 cudaError_t launch_compact_plan(const CompactParams& p, int n_streams, int32_t* first_moved,
                                 cudaStream_t st);
 cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap);
+cudaError_t launch_bounded_wait_selftest(int32_t* flag, uint32_t limit, int32_t* status,
+                                         cudaStream_t st);
 
 // ---- small device helpers ----------------------------------------------------------------
 #ifdef __CUDACC__
@@ -215,6 +217,24 @@ __device__ __forceinline__ void bulk_wait_all() {
 // mbarrier and within one kernel duration for a progress word; these limits are seconds)
 constexpr uint32_t kSpinLimit = 1u << 22;      // global-memory progress words
 constexpr uint32_t kMbarSpinLimit = 1u << 20;  // mbarrier phases (each poll may itself suspend)
+
+// Progress words in global memory (release / acquire at GPU scope) and the bounded wait on them.
+__device__ __forceinline__ uint32_t ld_acquire(const int32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(int32_t* p, uint32_t v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// false if *flag did not become `want` within `limit` polls
+__device__ __forceinline__ bool wait_progress_word(const int32_t* flag, uint32_t want, uint32_t limit) {
+    uint32_t spins = 0;
+    while (ld_acquire(flag) != want) {
+        if (++spins > limit) return false;
+    }
+    return true;
+}
 
 // Order-preserving map from fp32 bit patterns to unsigned integers: a larger key is a
 // larger score; negatives sort below non-negatives and -0 below +0.

@@ -44,15 +44,6 @@ struct StageInfo {
     uint32_t pad;
 };
 
-__device__ __forceinline__ uint32_t ld_acquire(const int32_t* p) {
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_release(int32_t* p, uint32_t v) {
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-
 // Lane 0 waits for the loads of chunk c, honours the plane's progress word and stores the
 // chunk.  Returns false (to all lanes) if a wait ran out.
 __device__ __forceinline__ bool store_chunk(uint64_t* full, StageInfo* info, char* buf, int64_t c,
@@ -63,15 +54,7 @@ __device__ __forceinline__ bool store_chunk(uint64_t* full, StageInfo* info, cha
         const uint32_t parity = (uint32_t)((c / stages) & 1);
         ok = mbar_wait_bounded(&full[stage], parity, kMbarSpinLimit);
         const StageInfo si = info[stage];
-        if (ok && si.wait_val != 0) {
-            uint32_t spins = 0;
-            while (ld_acquire(si.flag) != si.wait_val) {
-                if (++spins > kSpinLimit) {
-                    ok = false;
-                    break;
-                }
-            }
-        }
+        if (ok && si.wait_val != 0) ok = wait_progress_word(si.flag, si.wait_val, kSpinLimit);
         if (ok) {
             if (si.signal_val != 0) st_release(si.flag, si.signal_val);
             bulk_store(si.dst, buf + (size_t)stage * stage_bytes, si.bytes);
@@ -232,7 +215,21 @@ __global__ void compact_plan_kernel(const CompactParams p, int32_t* __restrict__
     }
 }
 
+// Polls a progress word nobody sets, with the same bounded wait the gather uses, and reports
+// the expiry through the status word: lets a caller check the time-out path on a healthy GPU.
+__global__ void bounded_wait_selftest_kernel(int32_t* flag, uint32_t never, uint32_t limit,
+                                             int32_t* status) {
+    if (!wait_progress_word(flag, never, limit)) atomicOr(status, SIRLLM_STATUS_TIMEOUT);
+}
+
 }  // namespace
+
+cudaError_t launch_bounded_wait_selftest(int32_t* flag, uint32_t limit, int32_t* status,
+                                         cudaStream_t st) {
+    // progress words always have their top bit set; 1 is a value none of them ever takes
+    bounded_wait_selftest_kernel<<<1, 1, 0, st>>>(flag, 1u, limit, status);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_compact_plan(const CompactParams& p, int n_streams, int32_t* first_moved,
                                 cudaStream_t st) {

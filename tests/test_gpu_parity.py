@@ -661,3 +661,20 @@ def test_compact_in_place_with_planes_cut_into_many_chained_segments():
     _compact_case(1, 2, 49152, 64, [30000], True, 22)
     # out of place with the same cut (no chain needed, all rows copied)
     _compact_case(2, 1, 20000, 128, [15000, 777], False, 23)
+
+
+def test_a_device_side_wait_that_runs_out_is_reported_not_hung():
+    # failure detection without a failure: the library's bounded wait polls a progress word that
+    # nothing sets, gives up, raises the status bit, and the context keeps working
+    w = wl.WORKLOADS["tiny"].scaled(n_layers=1, n_kv_heads=1, capacity=128, budget=64, n_recent=8,
+                                    new_tokens=40, vocab=501)
+    st = DeviceState(w)
+    B.sirllm_selftest_bounded_wait(st.cfg, st.ws, 2000)
+    assert B.sirllm_status(st.ws, clear=True) == B.STATUS_TIMEOUT
+    assert B.sirllm_status(st.ws) == 0
+    for r in range(3):                      # the same workspace still runs rounds correctly
+        st.fill_round(r)
+        st.step()
+    assert B.sirllm_status(st.ws) == 0
+    st.check_kv_by_content()
+    assert st.host_len == [64]
