@@ -5,9 +5,11 @@
 
 A step is one evicting round of the whole pass over one batch of synthetic input at steady
 state (live length = budget before the round's tokens arrive).  One JSON line is printed by
-rank 0.  Under torchrun every rank drives its own GPU with its own independent streams (the
+rank 0.  With N > 1 every rank drives its own GPU with its own independent streams (the
 pass shards by stream; there is no collective on the data path) and the line reports the
-whole job: weak scaling.
+whole job: weak scaling.  The N ranks come from torchrun (RANK / WORLD_SIZE in the
+environment) or, when the script is started plainly with --gpus N, from N child processes
+it starts itself, one per GPU.
 
 Timing: CUDA events on the launching stream, barrier + synchronize on both sides, max over
 ranks.  The K timed rounds run back to back; every round reads a logits tensor (>= 1 GB on
@@ -19,6 +21,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -441,6 +444,25 @@ def run_e2e(p: Pass, args, dist, world):
 # the oracle on the host cores: CPU baseline of the CUDA arm and the reference arm
 # --------------------------------------------------------------------------------------------
 
+def host_info() -> dict:
+    """The machine the oracle was timed on: logical cores, CPU model, memory."""
+    model, ram_gb = None, None
+    try:
+        with open("/proc/cpuinfo") as fh:
+            for line in fh:
+                if line.lower().startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+        with open("/proc/meminfo") as fh:
+            for line in fh:
+                if line.startswith("MemTotal"):
+                    ram_gb = round(int(line.split()[1]) / 2 ** 20, 1)
+                    break
+    except OSError:
+        pass
+    return {"nproc": os.cpu_count(), "cpu_model": model, "ram_gb": ram_gb}
+
+
 def oracle_rounds(p: Pass, rounds: int):
     """Times `rounds` full evicting rounds of the oracle, as it stands, on a host copy of the
     device state (1 thread)."""
@@ -467,7 +489,7 @@ def oracle_rounds(p: Pass, rounds: int):
     return {"value": round(rounds * S * M / dt, 1), "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": f"{rounds} full evicting rounds of {w.name} (all {S * M} tokens, all "
                       f"{2 * w.planes_per_stream * S} planes), {dt:.1f} s of CPU time",
-            "seconds_per_round": round(dt / rounds, 3)}
+            "seconds_per_round": round(dt / rounds, 3), "host": host_info()}
 
 
 def run_reference(args, rank, world):
@@ -532,10 +554,33 @@ def run_reference(args, rank, world):
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": config_dict(w, world),
             "cpu_baseline": {"value": round(value, 1), "unit": UNIT, "cores": 1, "kind": "oracle",
-                             "sample": sample},
+                             "sample": sample, "host": host_info()},
             "e2e": {"value": round(value, 1), "unit": UNIT, "h2d_bytes_per_step": 0,
                     "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
+
+
+def launch_ranks(n: int) -> int:
+    """Started plainly with --gpus N: run N copies of this script as ranks 0..N-1, one per GPU
+    (the environment torchrun would have set, rendezvous on 127.0.0.1), and wait for them.
+    Rank 0 prints the job's line on the inherited stdout."""
+    visible = torch.cuda.device_count()
+    if n > visible:
+        print(f"bench.py: --gpus {n} needs {n} visible CUDA devices, this machine shows {visible}; "
+              f"nothing was run", file=sys.stderr)
+        return 2
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    procs = []
+    for rank in range(n):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__), *sys.argv[1:]], env=env))
+    rc = 0
+    for proc in procs:
+        rc = max(rc, abs(proc.wait()))
+    return rc
 
 
 def main():
@@ -551,12 +596,21 @@ def main():
     ap.add_argument("--graph", action="store_true",
                     help="replay the timed rounds from a captured CUDA graph (launch-bound shapes)")
     args = ap.parse_args()
+    if args.gpus < 1:
+        ap.error("--gpus must be at least 1")
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    under_launcher = "WORLD_SIZE" in os.environ
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if under_launcher and world != args.gpus and rank == 0:
+        print(f"bench.py: --gpus {args.gpus} but the launcher started {world} ranks; reporting "
+              f"n_gpus = {world}", file=sys.stderr)
     if args.impl == "reference":
-        run_reference(args, rank, world)
+        # the oracle runs on the host cores of rank 0 alone, whatever N is
+        run_reference(args, rank, world if under_launcher else args.gpus)
+    elif not under_launcher and args.gpus > 1:
+        sys.exit(launch_ranks(args.gpus))
     else:
         run_ours(args, rank, world, local_rank)
 

@@ -17,9 +17,12 @@
  *     Calls validate their arguments on the host, enqueue work on that stream and
  *     return without synchronising (sirllm_status() is the exception).  Two calls
  *     that use the same workspace must be ordered on the same stream.
- *   - Return value: SIRLLM_OK or a negative SIRLLM_ERR_* code.  Nothing is
- *     enqueued when a negative code is returned.  Conditions only the device can
- *     see are OR-ed into a sticky status word in `ws` (SIRLLM_STATUS_* bits).
+ *   - Return value: SIRLLM_OK or a negative SIRLLM_ERR_* code.  Every argument check
+ *     runs on the host before the first copy or launch: when NULL, BAD_CONFIG, ALIGN or
+ *     TOO_LARGE is returned nothing was enqueued and no buffer was touched.
+ *     SIRLLM_ERR_CUDA reports a runtime call that failed, possibly part-way through the
+ *     call's sequence.  Conditions only the device can see are OR-ed into a sticky
+ *     status word in `ws` (SIRLLM_STATUS_* bits).
  *   - Layouts.  Logits: row-major rows of `vocab` elements, `logits_row_stride`
  *     elements apart; stream s owns rows [s*max_new, s*max_new + n_new[s]).
  *     K and V: each one contiguous array [n_streams][n_layers][n_kv_heads]
@@ -227,8 +230,8 @@ int sirllm_compact_kv(const sirllm_config *cfg, const void *k_src, const void *v
  * compacted with the same keep lists: the key now in slot j was written for position
  * keep_idx[s][j]; it is turned by (j - keep_idx[s][j]) positions, pair i of the row by the
  * angle shift * rope_base^(-2i/head_dim), so that it becomes the key of a token at position
- * j.  Rows that did not move are not touched.  Angles are evaluated in fp64, the rotation in
- * fp32, and each element is rounded once to the K dtype.  (A model that caches keys before
+ * j.  Rows that did not move are not touched.  Angles and the rotation are evaluated in fp64
+ * and each element is rounded once, from fp64, to the K dtype.  (A model that caches keys before
  * the rotary embedding needs no such call: slot order already is the position.)
  *   k         the K cache of sirllm_compact_kv, updated in place; head_dim % 16 == 0
  *   rope_base the base of the frequencies (10000, 500000, ...); layout: SIRLLM_ROPE_*

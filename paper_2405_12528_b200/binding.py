@@ -30,6 +30,7 @@ EXPORTS = ["sirllm_workspace_bytes", "sirllm_workspace_init", "sirllm_score", "s
            "sirllm_last_cuda_error"]
 
 _DTYPE_CODE = {torch.float32: F32, torch.bfloat16: BF16, torch.float16: F16}
+_KV = (torch.bfloat16, torch.float16)
 
 
 class SirllmError(RuntimeError):
@@ -135,31 +136,160 @@ def _check(rc: int) -> None:
         raise SirllmError(rc, detail)
 
 
-def _dev(t: Optional[torch.Tensor], dtype=None, name="tensor") -> Optional[int]:
-    if t is None:
-        return None
-    if not t.is_cuda:
-        raise SirllmError(ERR_NULL, f"{name} must be a CUDA tensor (there is no CPU path)")
-    if not t.is_contiguous():
-        raise SirllmError(ERR_ALIGN, f"{name} must be contiguous")
-    if dtype is not None and t.dtype not in (dtype if isinstance(dtype, tuple) else (dtype,)):
-        raise SirllmError(ERR_BAD_CONFIG, f"{name} has dtype {t.dtype}")
-    return t.data_ptr()
+class _Arg:
+    """One tensor argument and what the configuration demands of it.  The C side sees plain
+    pointers and no sizes, so every call checks ALL its arguments here first - dtype and
+    element count, then residence (right kind of memory, contiguous, on the current device) -
+    and only then hands out pointers."""
+
+    def __init__(self, t, dtype, name, numel=0, host=False):
+        self.t, self.dtype, self.name, self.numel, self.host = t, dtype, name, numel, host
+
+    def check_shape(self):
+        t = self.t
+        if t is None:
+            return
+        if self.dtype is not None and t.dtype not in (self.dtype if isinstance(self.dtype, tuple) else (self.dtype,)):
+            raise SirllmError(ERR_BAD_CONFIG, f"{self.name} has dtype {t.dtype}")
+        if t.numel() < self.numel:
+            raise SirllmError(ERR_BAD_CONFIG, f"{self.name} holds {t.numel()} elements, the "
+                                              f"configuration needs {self.numel}")
+
+    def check_residence(self):
+        t = self.t
+        if t is None:
+            return
+        if self.host:
+            if t.is_cuda or not t.is_contiguous():
+                raise SirllmError(ERR_ALIGN, f"{self.name} must be a contiguous host tensor")
+            return
+        if not t.is_cuda:
+            raise SirllmError(ERR_NULL, f"{self.name} must be a CUDA tensor (there is no CPU path)")
+        if not t.is_contiguous() and self.dtype is not None:
+            raise SirllmError(ERR_ALIGN, f"{self.name} must be contiguous")
+        if t.device.index != torch.cuda.current_device():
+            raise SirllmError(ERR_BAD_CONFIG, f"{self.name} lives on {t.device}, the current device "
+                                              f"is cuda:{torch.cuda.current_device()}")
+
+    def ptr(self):
+        return None if self.t is None else self.t.data_ptr()
 
 
-def _stream() -> int:
+def _dev(t, dtype=None, name="tensor", numel: int = 0) -> _Arg:
+    return _Arg(t, dtype, name, numel)
+
+
+def _call(fn, cfg, *args) -> None:
+    """Checks every tensor argument (shapes of all first, then residence), then calls ``fn``."""
+    for a in args:
+        if isinstance(a, _Arg):
+            a.check_shape()
+    for a in args:
+        if isinstance(a, _Arg):
+            a.check_residence()
+    raw = [a.ptr() if isinstance(a, _Arg) else _stream_handle() if isinstance(a, _CurrentStream) else a
+           for a in args]
+    _check(fn(ctypes.byref(cfg), *raw))
+
+
+class _CurrentStream:
+    """Placeholder for the current CUDA stream's handle, looked up after the argument checks."""
+
+
+def _stream() -> _CurrentStream:
+    return _CurrentStream()
+
+
+def _stream_handle() -> int:
     return torch.cuda.current_stream().cuda_stream
 
 
-def _logits_ptr(cfg: Config, logits: torch.Tensor) -> int:
-    if not logits.is_cuda:
-        raise SirllmError(ERR_NULL, "logits must be a CUDA tensor (there is no CPU path)")
-    if _DTYPE_CODE.get(logits.dtype) != cfg.logits_dtype:
-        raise SirllmError(ERR_BAD_CONFIG, f"logits dtype {logits.dtype} does not match the config")
-    if logits.stride(-1) != 1 or (logits.dim() >= 2 and logits.shape[-2] > 1
-                                  and logits.stride(-2) != cfg.logits_row_stride):
-        raise SirllmError(ERR_ALIGN, "logits rows must be logits_row_stride elements apart")
-    return logits.data_ptr()
+def _rows(cfg: Config) -> int:
+    return cfg.n_streams * cfg.max_new
+
+
+def _kv_numel(cfg: Config) -> int:
+    return cfg.n_streams * cfg.n_layers * cfg.n_kv_heads * cfg.capacity * cfg.head_dim
+
+
+class _KvArg(_Arg):
+    def __init__(self, cfg, t, name):
+        super().__init__(t, _KV, name, _kv_numel(cfg))
+        self.code = cfg.kv_dtype
+
+    def check_shape(self):
+        super().check_shape()
+        if self.t is not None and _DTYPE_CODE.get(self.t.dtype) != self.code:
+            raise SirllmError(ERR_BAD_CONFIG, f"{self.name} dtype {self.t.dtype} does not match the config")
+
+
+def _kv(cfg: Config, t, name) -> _Arg:
+    return _KvArg(cfg, t, name)
+
+
+def _ws(cfg: Config, ws) -> _Arg:
+    return _dev(ws, torch.uint8, "ws", sirllm_workspace_bytes(cfg))
+
+
+class _LogitsArg(_Arg):
+    """A logits matrix [>= rows, vocab] whose rows are logits_row_stride elements apart
+    (a column slice of a wider buffer is fine: only the last dimension must be dense)."""
+
+    def __init__(self, cfg, t, name="logits", host=False):
+        super().__init__(t, None, name, 0, host)
+        self.cfg = cfg
+
+    def check_shape(self):
+        cfg, t = self.cfg, self.t
+        if t is None:
+            return
+        if _DTYPE_CODE.get(t.dtype) != cfg.logits_dtype:
+            raise SirllmError(ERR_BAD_CONFIG, f"{self.name} dtype {t.dtype} does not match the config")
+        rows = _rows(cfg)
+        if t.dim() != 2 or t.shape[1] != cfg.vocab or t.shape[0] < rows:
+            raise SirllmError(ERR_BAD_CONFIG, f"{self.name} has shape {tuple(t.shape)}, the "
+                                              f"configuration needs [>= {rows}, {cfg.vocab}]")
+        if t.stride(1) != 1 or (t.shape[0] > 1 and t.stride(0) != cfg.logits_row_stride):
+            raise SirllmError(ERR_ALIGN, f"{self.name} rows must be logits_row_stride elements apart")
+
+    def check_residence(self):
+        if self.host and self.t is not None:
+            if self.t.is_cuda:
+                raise SirllmError(ERR_ALIGN, f"{self.name} must be a host tensor")
+            return
+        super().check_residence()
+
+
+def _logits(cfg: Config, logits) -> _Arg:
+    return _LogitsArg(cfg, logits)
+
+
+class _PairsArg(_Arg):
+    """Per-tile (max, sum exp) pairs [>= rows, n_tiles, 2], fp32, pairs contiguous."""
+
+    def __init__(self, cfg, t):
+        super().__init__(t, None, "pairs")
+        self.cfg = cfg
+
+    def check_shape(self):
+        t = self.t
+        if t is None:
+            raise SirllmError(ERR_NULL, "pairs is required")
+        if t.dtype != torch.float32:
+            raise SirllmError(ERR_BAD_CONFIG, "pairs must be float32")
+        if t.dim() != 3 or t.shape[2] != 2 or t.stride(2) != 1 or t.stride(1) != 2:
+            raise SirllmError(ERR_ALIGN, "pairs must be [rows, n_tiles, 2] with contiguous pairs")
+        if t.shape[0] < _rows(self.cfg):
+            raise SirllmError(ERR_BAD_CONFIG, f"pairs hold {t.shape[0]} rows, the configuration "
+                                              f"needs {_rows(self.cfg)}")
+
+    @property
+    def n_tiles(self) -> int:
+        return int(self.t.shape[1])
+
+    @property
+    def row_stride(self) -> int:
+        return int(self.t.stride(0) // 2 if self.t.shape[0] > 1 else self.t.shape[1])
 
 
 def sirllm_workspace_bytes(cfg: Config) -> int:
@@ -177,120 +307,100 @@ def new_workspace(cfg: Config, device="cuda") -> torch.Tensor:
 
 
 def sirllm_workspace_init(cfg: Config, ws: torch.Tensor) -> None:
-    _check(lib().sirllm_workspace_init(ctypes.byref(cfg), _dev(ws, torch.uint8, "ws"), _stream()))
+    _call(lib().sirllm_workspace_init, cfg, _ws(cfg, ws), _stream())
+
+
+def _score_args(cfg: Config, token_ids, n_new, out_entropy):
+    return (_dev(token_ids, torch.int32, "token_ids", _rows(cfg)),
+            _dev(n_new, torch.int32, "n_new", cfg.n_streams),
+            _dev(out_entropy, torch.float32, "out_entropy", _rows(cfg)))
 
 
 def sirllm_score(cfg: Config, logits, token_ids, n_new, out_entropy, ws) -> None:
-    _check(lib().sirllm_score(ctypes.byref(cfg), _logits_ptr(cfg, logits),
-                              _dev(token_ids, torch.int32, "token_ids"),
-                              _dev(n_new, torch.int32, "n_new"),
-                              _dev(out_entropy, torch.float32, "out_entropy"),
-                              _dev(ws, torch.uint8, "ws"), _stream()))
+    _call(lib().sirllm_score, cfg, _logits(cfg, logits), *_score_args(cfg, token_ids, n_new, out_entropy),
+          _ws(cfg, ws), _stream())
 
 
 def sirllm_score_static(cfg: Config, logits, token_ids, n_new, out_entropy, status=None) -> None:
     """``sirllm_score`` without a workspace: for callers that cannot allocate device memory
     (the scratch is a fixed array inside the library; at most 16384 logits rows per call,
     and calls that overlap on the GPU race).  ``status``: optional int32 device word."""
-    _check(lib().sirllm_score_static(ctypes.byref(cfg), _logits_ptr(cfg, logits),
-                                     _dev(token_ids, torch.int32, "token_ids"),
-                                     _dev(n_new, torch.int32, "n_new"),
-                                     _dev(out_entropy, torch.float32, "out_entropy"),
-                                     _dev(status, torch.int32, "status"), _stream()))
-
-
-def _pairs_args(pairs: torch.Tensor):
-    if pairs.dim() != 3 or pairs.shape[2] != 2 or pairs.stride(2) != 1 or pairs.stride(1) != 2:
-        raise SirllmError(ERR_ALIGN, "pairs must be [rows, n_tiles, 2] with contiguous pairs")
-    stride = pairs.stride(0) // 2 if pairs.shape[0] > 1 else pairs.shape[1]
-    if not pairs.is_cuda or pairs.dtype != torch.float32:
-        raise SirllmError(ERR_BAD_CONFIG, "pairs must be a float32 CUDA tensor")
-    return pairs.data_ptr(), int(pairs.shape[1]), int(stride)
+    _call(lib().sirllm_score_static, cfg, _logits(cfg, logits),
+          *_score_args(cfg, token_ids, n_new, out_entropy), _dev(status, torch.int32, "status", 1),
+          _stream())
 
 
 def sirllm_score_pairs(cfg: Config, pairs, target_logit, token_ids, n_new, out_entropy, ws) -> None:
     """Scores from per-tile ``(max, sum exp)`` pairs ``[rows, n_tiles, 2]`` and target logits."""
-    ptr, n_tiles, stride = _pairs_args(pairs)
-    _check(lib().sirllm_score_pairs(ctypes.byref(cfg), ptr, n_tiles, stride,
-                                    _dev(target_logit, torch.float32, "target_logit"),
-                                    _dev(token_ids, torch.int32, "token_ids"),
-                                    _dev(n_new, torch.int32, "n_new"),
-                                    _dev(out_entropy, torch.float32, "out_entropy"),
-                                    _dev(ws, torch.uint8, "ws"), _stream()))
+    pa = _PairsArg(cfg, pairs)
+    pa.check_shape()
+    _call(lib().sirllm_score_pairs, cfg, pa, pa.n_tiles, pa.row_stride,
+          _dev(target_logit, torch.float32, "target_logit", _rows(cfg)),
+          *_score_args(cfg, token_ids, n_new, out_entropy), _ws(cfg, ws), _stream())
+
+
+def _state_args(cfg: Config, scores, serial, live_len, decay):
+    per_slot = cfg.n_streams * cfg.capacity
+    return (_dev(scores, torch.float32, "scores", per_slot),
+            _dev(serial, torch.int64, "serial", per_slot),
+            _dev(live_len, torch.int32, "live_len", cfg.n_streams),
+            _dev(decay, torch.float32, "decay", cfg.n_streams))
+
+
+def _keep_args(cfg: Config, keep_idx, n_keep):
+    return (_dev(keep_idx, torch.int32, "keep_idx", cfg.n_streams * cfg.threshold),
+            _dev(n_keep, torch.int32, "n_keep", cfg.n_streams))
+
+
+def _round_args(cfg: Config, token_ids, n_new, scores, serial, live_len, decay, k, v, keep_idx, n_keep,
+                new_entropy, ws):
+    """The arguments sirllm_step, _step_pairs, _step_phases and _step_host share, in ABI order."""
+    ids, nn, ent = _score_args(cfg, token_ids, n_new, new_entropy)
+    return (ids, nn) + _state_args(cfg, scores, serial, live_len, decay) + \
+        (_kv(cfg, k, "k"), _kv(cfg, v, "v")) + _keep_args(cfg, keep_idx, n_keep) + (ent, _ws(cfg, ws))
 
 
 def sirllm_step_pairs(cfg: Config, pairs, target_logit, token_ids, n_new, scores, serial, live_len,
                       decay, k, v, keep_idx, n_keep, new_entropy, ws) -> None:
-    ptr, n_tiles, stride = _pairs_args(pairs)
-    _check(lib().sirllm_step_pairs(ctypes.byref(cfg), ptr, n_tiles, stride,
-                                   _dev(target_logit, torch.float32, "target_logit"),
-                                   _dev(token_ids, torch.int32, "token_ids"),
-                                   _dev(n_new, torch.int32, "n_new"),
-                                   _dev(scores, torch.float32, "scores"),
-                                   _dev(serial, torch.int64, "serial"),
-                                   _dev(live_len, torch.int32, "live_len"),
-                                   _dev(decay, torch.float32, "decay"),
-                                   _dev(k, _KV, "k"), _dev(v, _KV, "v"),
-                                   _dev(keep_idx, torch.int32, "keep_idx"),
-                                   _dev(n_keep, torch.int32, "n_keep"),
-                                   _dev(new_entropy, torch.float32, "new_entropy"),
-                                   _dev(ws, torch.uint8, "ws"), _stream()))
+    pa = _PairsArg(cfg, pairs)
+    pa.check_shape()
+    _call(lib().sirllm_step_pairs, cfg, pa, pa.n_tiles, pa.row_stride,
+          _dev(target_logit, torch.float32, "target_logit", _rows(cfg)),
+          *_round_args(cfg, token_ids, n_new, scores, serial, live_len, decay, k, v, keep_idx, n_keep,
+                       new_entropy, ws), _stream())
 
 
 def sirllm_decay_select(cfg: Config, scores, serial, live_len, decay, keep_idx, n_keep,
                         compact_scores, ws) -> None:
-    _check(lib().sirllm_decay_select(ctypes.byref(cfg), _dev(scores, torch.float32, "scores"),
-                                     _dev(serial, torch.int64, "serial"),
-                                     _dev(live_len, torch.int32, "live_len"),
-                                     _dev(decay, torch.float32, "decay"),
-                                     _dev(keep_idx, torch.int32, "keep_idx"),
-                                     _dev(n_keep, torch.int32, "n_keep"),
-                                     int(bool(compact_scores)), _dev(ws, torch.uint8, "ws"), _stream()))
+    _call(lib().sirllm_decay_select, cfg, *_state_args(cfg, scores, serial, live_len, decay),
+          *_keep_args(cfg, keep_idx, n_keep), int(bool(compact_scores)), _ws(cfg, ws), _stream())
 
 
 def sirllm_keep_policy(cfg: Config, policy: int, live_len, seed: int, rnd: int, stream_base: int,
                        keep_idx, n_keep, ws) -> None:
     """Keep lists of StreamLLM / RandomLLM / IntervalLLM (``POLICY_*``) for ``sirllm_compact_kv``."""
-    _check(lib().sirllm_keep_policy(ctypes.byref(cfg), int(policy), _dev(live_len, torch.int32, "live_len"),
-                                    int(seed), int(rnd), int(stream_base),
-                                    _dev(keep_idx, torch.int32, "keep_idx"),
-                                    _dev(n_keep, torch.int32, "n_keep"),
-                                    _dev(ws, torch.uint8, "ws"), _stream()))
-
-
-_KV = (torch.bfloat16, torch.float16)
+    _call(lib().sirllm_keep_policy, cfg, int(policy), _dev(live_len, torch.int32, "live_len", cfg.n_streams),
+          int(seed), int(rnd), int(stream_base), *_keep_args(cfg, keep_idx, n_keep), _ws(cfg, ws),
+          _stream())
 
 
 def sirllm_rerotate_keys(cfg: Config, k, keep_idx, n_keep, rope_base: float, layout: int) -> None:
     """Turns the moved rows of a compacted post-rotary K cache to their new positions."""
-    _check(lib().sirllm_rerotate_keys(ctypes.byref(cfg), _dev(k, _KV, "k"),
-                                      _dev(keep_idx, torch.int32, "keep_idx"),
-                                      _dev(n_keep, torch.int32, "n_keep"), float(rope_base),
-                                      int(layout), _stream()))
+    _call(lib().sirllm_rerotate_keys, cfg, _kv(cfg, k, "k"), *_keep_args(cfg, keep_idx, n_keep),
+          float(rope_base), int(layout), _stream())
 
 
 def sirllm_compact_kv(cfg: Config, k_src, v_src, k_dst, v_dst, keep_idx, n_keep, ws) -> None:
-    _check(lib().sirllm_compact_kv(ctypes.byref(cfg), _dev(k_src, _KV, "k_src"), _dev(v_src, _KV, "v_src"),
-                                   _dev(k_dst, _KV, "k_dst"), _dev(v_dst, _KV, "v_dst"),
-                                   _dev(keep_idx, torch.int32, "keep_idx"),
-                                   _dev(n_keep, torch.int32, "n_keep"),
-                                   _dev(ws, torch.uint8, "ws"), _stream()))
+    _call(lib().sirllm_compact_kv, cfg, _kv(cfg, k_src, "k_src"), _kv(cfg, v_src, "v_src"),
+          _kv(cfg, k_dst, "k_dst"), _kv(cfg, v_dst, "v_dst"), *_keep_args(cfg, keep_idx, n_keep),
+          _ws(cfg, ws), _stream())
 
 
 def sirllm_step(cfg: Config, logits, token_ids, n_new, scores, serial, live_len, decay, k, v,
                 keep_idx, n_keep, new_entropy, ws) -> None:
-    _check(lib().sirllm_step(ctypes.byref(cfg), _logits_ptr(cfg, logits),
-                             _dev(token_ids, torch.int32, "token_ids"),
-                             _dev(n_new, torch.int32, "n_new"),
-                             _dev(scores, torch.float32, "scores"),
-                             _dev(serial, torch.int64, "serial"),
-                             _dev(live_len, torch.int32, "live_len"),
-                             _dev(decay, torch.float32, "decay"),
-                             _dev(k, _KV, "k"), _dev(v, _KV, "v"),
-                             _dev(keep_idx, torch.int32, "keep_idx"),
-                             _dev(n_keep, torch.int32, "n_keep"),
-                             _dev(new_entropy, torch.float32, "new_entropy"),
-                             _dev(ws, torch.uint8, "ws"), _stream()))
+    _call(lib().sirllm_step, cfg, _logits(cfg, logits),
+          *_round_args(cfg, token_ids, n_new, scores, serial, live_len, decay, k, v, keep_idx, n_keep,
+                       new_entropy, ws), _stream())
 
 
 def sirllm_step_phases(cfg: Config, logits, token_ids, n_new, scores, serial, live_len, decay, k, v,
@@ -302,28 +412,13 @@ def sirllm_step_phases(cfg: Config, logits, token_ids, n_new, scores, serial, li
         if not ev.cuda_event:          # torch creates the handle lazily, on first record
             ev.record()
         handles[i] = ev.cuda_event
-    _check(lib().sirllm_step_phases(ctypes.byref(cfg), _logits_ptr(cfg, logits),
-                                    _dev(token_ids, torch.int32, "token_ids"),
-                                    _dev(n_new, torch.int32, "n_new"),
-                                    _dev(scores, torch.float32, "scores"),
-                                    _dev(serial, torch.int64, "serial"),
-                                    _dev(live_len, torch.int32, "live_len"),
-                                    _dev(decay, torch.float32, "decay"),
-                                    _dev(k, _KV, "k"), _dev(v, _KV, "v"),
-                                    _dev(keep_idx, torch.int32, "keep_idx"),
-                                    _dev(n_keep, torch.int32, "n_keep"),
-                                    _dev(new_entropy, torch.float32, "new_entropy"),
-                                    _dev(ws, torch.uint8, "ws"), _stream(), handles))
+    _call(lib().sirllm_step_phases, cfg, _logits(cfg, logits),
+          *_round_args(cfg, token_ids, n_new, scores, serial, live_len, decay, k, v, keep_idx, n_keep,
+                       new_entropy, ws), _stream(), handles)
 
 
-def _host(t: Optional[torch.Tensor], dtype=None, name="tensor") -> Optional[int]:
-    if t is None:
-        return None
-    if t.is_cuda or not t.is_contiguous():
-        raise SirllmError(ERR_ALIGN, f"{name} must be a contiguous host tensor")
-    if dtype is not None and t.dtype not in (dtype if isinstance(dtype, tuple) else (dtype,)):
-        raise SirllmError(ERR_BAD_CONFIG, f"{name} has dtype {t.dtype}")
-    return t.data_ptr()
+def _host(t, dtype=None, name="tensor", numel: int = 0) -> _Arg:
+    return _Arg(t, dtype, name, numel, host=True)
 
 
 def sirllm_step_host(cfg: Config, h_logits, h_token_ids, h_n_new, h_new_k, h_new_v, h_live_len,
@@ -331,31 +426,31 @@ def sirllm_step_host(cfg: Config, h_logits, h_token_ids, h_n_new, h_new_k, h_new
                      keep_idx, n_keep, new_entropy, h_keep_idx, h_n_keep, h_new_entropy, ws) -> None:
     """One round with HOST inputs and outputs (``h_*`` are CPU tensors, ideally pinned);
     the results are valid after ``torch.cuda.current_stream().synchronize()``."""
-    ldt = {F32: torch.float32, BF16: torch.bfloat16}[cfg.logits_dtype]
-    _check(lib().sirllm_step_host(
-        ctypes.byref(cfg), _host(h_logits, ldt, "h_logits"), _host(h_token_ids, torch.int32, "h_token_ids"),
-        _host(h_n_new, torch.int32, "h_n_new"), _host(h_new_k, _KV, "h_new_k"),
-        _host(h_new_v, _KV, "h_new_v"), _host(h_live_len, torch.int32, "h_live_len"),
-        _logits_ptr(cfg, d_logits), _dev(d_token_ids, torch.int32, "d_token_ids"),
-        _dev(d_n_new, torch.int32, "d_n_new"), _dev(scores, torch.float32, "scores"),
-        _dev(serial, torch.int64, "serial"), _dev(live_len, torch.int32, "live_len"),
-        _dev(decay, torch.float32, "decay"), _dev(k, _KV, "k"), _dev(v, _KV, "v"),
-        _dev(keep_idx, torch.int32, "keep_idx"), _dev(n_keep, torch.int32, "n_keep"),
-        _dev(new_entropy, torch.float32, "new_entropy"), _host(h_keep_idx, torch.int32, "h_keep_idx"),
-        _host(h_n_keep, torch.int32, "h_n_keep"), _host(h_new_entropy, torch.float32, "h_new_entropy"),
-        _dev(ws, torch.uint8, "ws"), _stream()))
+    rows, S = _rows(cfg), cfg.n_streams
+    new_rows = S * cfg.n_layers * cfg.n_kv_heads * cfg.max_new * cfg.head_dim
+    rest = _round_args(cfg, d_token_ids, d_n_new, scores, serial, live_len, decay, k, v, keep_idx,
+                       n_keep, new_entropy, ws)
+    _call(lib().sirllm_step_host, cfg, _LogitsArg(cfg, h_logits, "h_logits", host=True),
+          _host(h_token_ids, torch.int32, "h_token_ids", rows), _host(h_n_new, torch.int32, "h_n_new", S),
+          _host(h_new_k, _KV, "h_new_k", new_rows), _host(h_new_v, _KV, "h_new_v", new_rows),
+          _host(h_live_len, torch.int32, "h_live_len", S), _LogitsArg(cfg, d_logits, "d_logits"),
+          *rest[:-1], _host(h_keep_idx, torch.int32, "h_keep_idx", S * cfg.threshold),
+          _host(h_n_keep, torch.int32, "h_n_keep", S),
+          _host(h_new_entropy, torch.float32, "h_new_entropy", rows), rest[-1], _stream())
 
 
 def sirllm_selftest_bounded_wait(cfg: Config, ws: torch.Tensor, polls: int = 2000) -> None:
     """Lets one device-side bounded wait run out on purpose (raises STATUS_TIMEOUT in ``ws``)."""
-    _check(lib().sirllm_selftest_bounded_wait(ctypes.byref(cfg), _dev(ws, torch.uint8, "ws"),
-                                              int(polls), _stream()))
+    _call(lib().sirllm_selftest_bounded_wait, cfg, _ws(cfg, ws), int(polls), _stream())
 
 
 def sirllm_status(ws: torch.Tensor, clear: bool = False) -> int:
     """Synchronises the current stream and returns the device status word."""
     out = ctypes.c_int32(0)
-    _check(lib().sirllm_status(_dev(ws, torch.uint8, "ws"), _stream(), ctypes.byref(out), int(clear)))
+    arg = _dev(ws, torch.uint8, "ws", 4)
+    arg.check_shape()
+    arg.check_residence()
+    _check(lib().sirllm_status(arg.ptr(), _stream_handle(), ctypes.byref(out), int(clear)))
     return out.value
 
 

@@ -142,6 +142,7 @@ static SelectParams select_params(const sirllm_config& c, const WorkspaceLayout&
     p.first_moved = (int32_t*)((char*)ws + L.first_moved_off);
     p.status = (int32_t*)ws;
     p.epoch = (int32_t*)ws + 1;
+    p.ticket = (unsigned long long*)ws + 1;
     p.capacity = c.capacity;
     p.budget = c.budget;
     p.n_sink = c.n_sink;
@@ -217,6 +218,7 @@ static int compact_params(const sirllm_config& c, const WorkspaceLayout& L, cons
     p.first_moved = (int32_t*)((char*)ws + L.first_moved_off);
     p.status = (int32_t*)ws;
     p.epoch = (int32_t*)ws + 1;
+    p.ticket = (unsigned long long*)ws + 1;
     p.plane_flags = (int32_t*)((char*)ws + L.plane_flags_off);
     p.planes_per_stream = c.n_layers * c.n_kv_heads;
     p.planes_per_tensor = (int64_t)c.n_streams * p.planes_per_stream;
@@ -283,10 +285,21 @@ static PairScoreParams pair_params(const sirllm_config& c, const ScoreSource& sr
     return pp;
 }
 
-static int step_impl(const sirllm_config* cfg, const ScoreSource& src, const int32_t* token_ids,
-                     const int32_t* n_new, float* scores, int64_t* serial, int32_t* live_len,
-                     const float* decay, void* k, void* v, int32_t* keep_idx, int32_t* n_keep,
-                     float* new_entropy, void* ws, void* cuda_stream, void** ev) {
+// Everything one round launches, checked and laid out before anything is enqueued.
+struct StepPlan {
+    bool from_pairs;
+    ScoreParams sc;
+    PairScoreParams pp;
+    SelectParams sp;
+    CompactParams cp;
+    int n_streams;
+};
+
+// Host-side validation of a whole round; touches no device and enqueues nothing.
+static int step_prepare(const sirllm_config* cfg, const ScoreSource& src, const int32_t* token_ids,
+                        const int32_t* n_new, float* scores, int64_t* serial, int32_t* live_len,
+                        const float* decay, void* k, void* v, int32_t* keep_idx, int32_t* n_keep,
+                        float* new_entropy, void* ws, StepPlan* plan) {
     int rc = validate_config(cfg);
     if (rc != SIRLLM_OK) return rc;
     if (!token_ids || !scores || !live_len || !decay || !ws) return SIRLLM_ERR_NULL;
@@ -298,39 +311,57 @@ static int step_impl(const sirllm_config* cfg, const ScoreSource& src, const int
         return rc;
     }
     const WorkspaceLayout L = workspace_layout(*cfg);
-    SelectParams sp = select_params(*cfg, L, scores, serial, live_len, decay, keep_idx, n_keep, ws);
-    ScoreParams sc = score_params(*cfg, L, src.logits, token_ids, n_new, ws);
-    sc.out_entropy = new_entropy;
-    sc.scores = scores;
-    sc.live_len = live_len;
-    PairScoreParams pp = pair_params(*cfg, src, token_ids, n_new, ws);
-    pp.out_entropy = new_entropy;
-    pp.scores = scores;
-    pp.live_len = live_len;
-    sp.n_new = n_new;
-    sp.max_new = cfg->max_new;
-    sp.compact_scores = 1;
-    sp.score_new = 1;
-    CompactParams cp;
-    if ((rc = compact_params(*cfg, L, k, v, k, v, sp.keep_idx, sp.n_keep, ws, &cp)) != SIRLLM_OK)
-        return rc;
-    cudaStream_t st = (cudaStream_t)cuda_stream;
+    plan->from_pairs = src.pairs != nullptr;
+    plan->n_streams = cfg->n_streams;
+    plan->sp = select_params(*cfg, L, scores, serial, live_len, decay, keep_idx, n_keep, ws);
+    plan->sc = score_params(*cfg, L, src.logits, token_ids, n_new, ws);
+    plan->sc.out_entropy = new_entropy;
+    plan->sc.scores = scores;
+    plan->sc.live_len = live_len;
+    plan->pp = pair_params(*cfg, src, token_ids, n_new, ws);
+    plan->pp.out_entropy = new_entropy;
+    plan->pp.scores = scores;
+    plan->pp.live_len = live_len;
+    plan->sp.n_new = n_new;
+    plan->sp.max_new = cfg->max_new;
+    plan->sp.compact_scores = 1;
+    plan->sp.score_new = 1;
+    return compact_params(*cfg, L, k, v, k, v, plan->sp.keep_idx, plan->sp.n_keep, ws, &plan->cp);
+}
+
+// The round's three launches (with `ev`: four event records around them, and no overlap
+// between the kernels so that the events separate the phases).
+static int step_enqueue(const StepPlan& plan, cudaStream_t st, void** ev) {
     cudaError_t e;
 #define SIRLLM_MARK(i)                                                        \
     if (ev && (e = cudaEventRecord((cudaEvent_t)ev[i], st)) != cudaSuccess) \
         return cuda_fail(e, "cudaEventRecord");
     SIRLLM_MARK(0)
-    e = src.pairs ? launch_score_pairs(pp, st) : launch_score(sc, st);
+    e = plan.from_pairs ? launch_score_pairs(plan.pp, st) : launch_score(plan.sc, st);
     if (e != cudaSuccess) return cuda_fail(e, "score");
     SIRLLM_MARK(1)
-    e = launch_select(sp, cfg->n_streams, st, ev == nullptr);
+    // the selection kernel reads the caller's buffers before it waits for its predecessor: it may
+    // only overlap the scorer, which itself started after all earlier work on the stream
+    const bool scored = (int64_t)plan.n_streams * plan.sp.max_new > 0;
+    e = launch_select(plan.sp, plan.n_streams, st, ev == nullptr && scored);
     if (e != cudaSuccess) return cuda_fail(e, "select");
     SIRLLM_MARK(2)
-    e = launch_compact(cp, st, ev == nullptr);
+    e = launch_compact(plan.cp, st, ev == nullptr);
     if (e != cudaSuccess) return cuda_fail(e, "compact");
     SIRLLM_MARK(3)
 #undef SIRLLM_MARK
     return SIRLLM_OK;
+}
+
+static int step_impl(const sirllm_config* cfg, const ScoreSource& src, const int32_t* token_ids,
+                     const int32_t* n_new, float* scores, int64_t* serial, int32_t* live_len,
+                     const float* decay, void* k, void* v, int32_t* keep_idx, int32_t* n_keep,
+                     float* new_entropy, void* ws, void* cuda_stream, void** ev) {
+    StepPlan plan;
+    const int rc = step_prepare(cfg, src, token_ids, n_new, scores, serial, live_len, decay, k, v,
+                                keep_idx, n_keep, new_entropy, ws, &plan);
+    if (rc != SIRLLM_OK) return rc;
+    return step_enqueue(plan, (cudaStream_t)cuda_stream, ev);
 }
 
 int sirllm_step(const sirllm_config* cfg, const void* logits, const int32_t* token_ids,
@@ -406,6 +437,17 @@ int sirllm_step_host(const sirllm_config* cfg, const void* h_logits, const int32
         return SIRLLM_ERR_NULL;
     if ((h_new_k != nullptr && k == nullptr) || (h_new_v != nullptr && v == nullptr))
         return SIRLLM_ERR_NULL;
+    // every check comes before the first copy: a refused call leaves the device untouched
+    for (int s = 0; s < cfg->n_streams; ++s) {
+        if (h_n_new[s] < 0 || h_n_new[s] > cfg->max_new || h_live_len[s] < 0)
+            return SIRLLM_ERR_BAD_CONFIG;
+    }
+    ScoreSource src;
+    src.logits = d_logits;
+    StepPlan plan;
+    rc = step_prepare(cfg, src, d_token_ids, d_n_new, scores, serial, live_len, decay, k, v,
+                      keep_idx, n_keep, new_entropy, ws, &plan);
+    if (rc != SIRLLM_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const size_t es = (size_t)logits_elem_bytes(cfg->logits_dtype);
     const size_t row_bytes = (size_t)cfg->head_dim * 2;
@@ -413,8 +455,7 @@ int sirllm_step_host(const sirllm_config* cfg, const void* h_logits, const int32
     cudaError_t e;
     for (int s = 0; s < cfg->n_streams; ++s) {
         const int T = h_n_new[s], l = h_live_len[s];
-        if (T < 0 || T > cfg->max_new || l < 0) return SIRLLM_ERR_BAD_CONFIG;
-        if (T == 0 || l + T > cfg->capacity) continue;  // the device skips and flags an overflow
+        if (T == 0 || l > cfg->capacity - T) continue;  // the device skips and flags an overflow
         const size_t row0 = (size_t)s * cfg->max_new;
         if (cfg->logits_row_stride == cfg->vocab) {
             e = cudaMemcpyAsync((char*)d_logits + row0 * cfg->vocab * es,
@@ -445,11 +486,7 @@ int sirllm_step_host(const sirllm_config* cfg, const void* h_logits, const int32
     if (e != cudaSuccess) return cuda_fail(e, "ids H2D");
     e = cudaMemcpyAsync(d_n_new, h_n_new, (size_t)cfg->n_streams * 4, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(e, "n_new H2D");
-    ScoreSource src;
-    src.logits = d_logits;
-    rc = step_impl(cfg, src, d_token_ids, d_n_new, scores, serial, live_len, decay, k, v,
-                   keep_idx, n_keep, new_entropy, ws, cuda_stream, nullptr);
-    if (rc != SIRLLM_OK) return rc;
+    if ((rc = step_enqueue(plan, st, nullptr)) != SIRLLM_OK) return rc;
     e = cudaMemcpyAsync(h_keep_idx, keep_idx, (size_t)cfg->n_streams * cfg->threshold * 4,
                         cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return cuda_fail(e, "keep D2H");

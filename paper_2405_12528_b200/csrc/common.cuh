@@ -9,7 +9,8 @@
 namespace sirllm {
 
 // ---- workspace layout (device memory owned by the caller) -------------------------------
-//   [0, 256)                              header: int32 status word, int32 compaction epoch
+//   [0, 256)                              header: int32 status word, int32 compaction epoch,
+//                                         uint64 ticket counter of the KV gather's work units
 //   plane_flags[2*n_streams*planes]       progress of a plane split across several workers
 //   first_moved[n_streams]                first slot whose row changes place when compacting
 //   n_keep_fallback[n_streams]            used when the caller passes no n_keep
@@ -32,7 +33,6 @@ struct WorkspaceLayout {
 
 constexpr int kScoreCtaVecs = 4096;  // 16-byte vectors of one logits row per CTA: 64 KB, shared
                                      // by 4 warps (16 KB each) or, in small grids, 8 or 16
-constexpr int kListMax = 256;  // keys ranked directly once a radix bin holds no more
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int logits_elem_bytes(int dtype) { return dtype == SIRLLM_F32 ? 4 : 2; }
@@ -82,6 +82,7 @@ struct SelectParams {
     int32_t* first_moved;
     int32_t* status;
     int32_t* epoch;
+    unsigned long long* ticket;  // hand-out counter of the gather that follows: reset with the epoch
     int32_t capacity, budget, n_sink, n_recent, threshold;
     int32_t compact_scores;  // also gather scores / serial and commit live_len
     int32_t score_new;       // the round's new scores were appended behind live_len by the scorer
@@ -111,6 +112,7 @@ struct CompactParams {
     const int32_t* first_moved;
     int32_t* status;
     int32_t* epoch;        // bumped once per compaction by the kernel that precedes it
+    unsigned long long* ticket;  // next work unit to hand out; zeroed by the same kernel
     int32_t* plane_flags;  // [tensors * planes_per_tensor]
     int64_t planes_per_tensor;  // n_streams * n_layers * n_kv_heads
     int32_t planes_per_stream;

@@ -16,13 +16,16 @@
 // landed, and later chunks only read rows behind everything stored so far.
 //
 // To fill all SMs evenly, the moved rows of a plane are cut into `split` segments that
-// different workers take (segment-major order, so a plane's earlier segments are handed
-// out long before its later ones).  A segment may store only after every earlier segment
-// of its plane has landed all its loads; that is tracked by one progress word per plane
-// (epoch * 64 + finished segments) written with release and polled with acquire, with an
-// iteration limit.  All workers are resident at once (one CTA per SM at most), and a
-// worker only ever waits for a unit that precedes its own in the hand-out order, so the
-// waits cannot form a cycle.
+// different workers take.  Work units (plane, segment) are numbered segment-major, so a
+// plane's earlier segments come long before its later ones, and are handed out in that order
+// through one ticket counter in the workspace: a worker that is ready draws the next number.
+// A segment may store only after every earlier segment of its plane has landed all its loads;
+// that is tracked by one progress word per plane (epoch * 64 + finished segments) written
+// with release and polled with acquire, with an iteration limit.  A worker only ever waits
+// for a unit with a smaller number than its own, and every smaller number was drawn by a
+// worker that is running (it drew the number itself), so by induction the waits end whatever
+// number of CTAs the device keeps resident at once; the hand-out also evens out SMs that run
+// at different speeds.
 #include "common.cuh"
 
 namespace sirllm {
@@ -34,6 +37,7 @@ constexpr int kStoreSlack = 1;  // bulk stores that may still be reading shared 
 constexpr int kMaxStages = 12;
 constexpr int kMaxSplit = 32;
 constexpr int kIdxAhead = 4;  // chunks whose source indices are fetched ahead
+constexpr int kMaxWorkers = 4;  // worker warps per CTA
 
 struct StageInfo {
     char* dst;           // destination of the chunk held by the stage
@@ -64,7 +68,7 @@ __device__ __forceinline__ bool store_chunk(uint64_t* full, StageInfo* info, cha
     return __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
 }
 
-__global__ void __launch_bounds__(256, 1)
+__global__ void __launch_bounds__(kMaxWorkers * 32, 1)
 compact_kernel(const CompactParams p, const int stages, const int units_base, const int split) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int n_workers = blockDim.x >> 5;
@@ -88,14 +92,18 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
 
     const uint32_t epoch_base = ((uint32_t)*p.epoch << 6) | 0x80000000u;  // never 0
     const int lead = stages - 1 - kStoreSlack;  // chunks whose loads run ahead of the stores
-    const int64_t g = (int64_t)blockIdx.x * n_workers + wid;
-    const int64_t G = (int64_t)gridDim.x * n_workers;
     const int64_t n_units = (int64_t)units_base * split;
     int64_t it = 0;      // chunks whose loads were issued
     int64_t stored = 0;  // chunks whose store was issued
     bool alive = true;
 
-    for (int64_t u = g; u < n_units && alive; u += G) {
+    // the next unit's number is drawn while the current unit is being moved
+    unsigned long long drawn = 0;
+    if (lane == 0) drawn = atomicAdd(p.ticket, 1ull);
+    while (alive) {
+        const int64_t u = (int64_t)__shfl_sync(0xFFFFFFFFu, drawn, 0);
+        if (u >= n_units) break;
+        if (lane == 0) drawn = atomicAdd(p.ticket, 1ull);
         const int h = (int)(u / units_base);  // segment of the plane's moved rows
         const int r = (int)(u - (int64_t)h * units_base);
         const int tensor = (int)(r / p.planes_per_tensor);
@@ -181,7 +189,13 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
         ++stored;
     }
     if (lane == 0) {
-        if (!alive) atomicOr(p.status, SIRLLM_STATUS_TIMEOUT);
+        if (!alive) {
+            // a wait ran out: nothing more is stored, but the bulk loads already issued still
+            // write into this CTA's shared memory - let them land (bounded) before leaving
+            atomicOr(p.status, SIRLLM_STATUS_TIMEOUT);
+            for (int64_t c = max(stored - 1, (int64_t)0); c < it; ++c)
+                (void)mbar_wait_bounded(&full[c % stages], (uint32_t)((c / stages) & 1), kMbarSpinLimit);
+        }
         bulk_wait_all();
     }
 }
@@ -195,7 +209,10 @@ __global__ void compact_plan_kernel(const CompactParams p, int32_t* __restrict__
     if (threadIdx.x == 0) {
         sh_first = n;
         sh_bad = (p.n_keep[s] < 0 || p.n_keep[s] > p.keep_stride) ? 1 : 0;
-        if (s == 0) *p.epoch += 1;  // a new compaction follows
+        if (s == 0) {  // a new compaction follows
+            *p.epoch += 1;
+            *p.ticket = 0ull;
+        }
     }
     __syncthreads();
     for (int j = threadIdx.x; j < n; j += blockDim.x) {
@@ -260,10 +277,11 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     if (e != cudaSuccess) return e;
 
-    // ring geometry: as many workers per SM as fit with at least 6 stages each (at most 8)
+    // ring geometry: kMaxWorkers workers per CTA with 6 to 8 stages each; fewer workers, then
+    // fewer stages (at least 4), when the rows are too wide for that
     const size_t stage_bytes = (size_t)kChunkRows * p.row_bytes;
     const size_t budget = (size_t)smem_max - 2048;
-    int workers = 4, stages = 6;
+    int workers = kMaxWorkers, stages = 6;
     while (workers > 1 && (size_t)workers * stages * stage_bytes > budget) --workers;
     while (stages > 4 && (size_t)workers * stages * stage_bytes > budget) --stages;
     if ((size_t)workers * stages * stage_bytes > budget) return cudaErrorInvalidValue;
@@ -274,9 +292,16 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     e = cudaFuncSetAttribute(compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
 
-    // one CTA per SM at most (all workers resident); cut planes into segments so that the
-    // units spread evenly over the workers: fewest idle worker-rounds, then fewest segments
-    const int64_t slots = (int64_t)n_sm * workers;
+    // a persistent grid: as many CTAs as the device keeps resident at once (the ring fills an
+    // SM's shared memory, so one per SM), fewer when there is less work
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compact_kernel, workers * 32, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+    const int64_t resident = (int64_t)n_sm * per_sm;
+    // cut planes into segments so that the units spread evenly over the workers: fewest idle
+    // worker-rounds, then fewest segments
+    const int64_t slots = resident * workers;
     int split = 1;
     if (units_base < 8 * slots) {
         double best = -1.0;
@@ -291,8 +316,8 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
         }
     }
     const int64_t n_units = (int64_t)units_base * split;
-    const int grid = (int)((n_units + workers - 1) / workers < n_sm ? (n_units + workers - 1) / workers
-                                                                    : n_sm);
+    const int64_t want = (n_units + workers - 1) / workers;
+    const int grid = (int)(want < resident ? want : resident);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)workers * 32);

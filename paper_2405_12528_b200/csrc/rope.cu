@@ -7,7 +7,12 @@
 // Bound by HBM traffic on the moved rows of the K planes (read once, written once).  The
 // angles depend on (stream, slot, pair) only, so a thread computes its eight (cos, sin) once -
 // in fp64, the shift can be thousands of positions - and reuses them for every K plane of its
-// group; per plane it moves two 16-byte vectors, rotates in fp32 and rounds once to bf16/fp16.
+// group; per plane it moves two 16-byte vectors.  The rotation itself is also carried out in
+// fp64 and every element is rounded ONCE, from fp64, to bf16/fp16: the result is the exactly
+// rotated value rounded to nearest even (an fp32 rotation loses the low bits of the products
+// where x cos - y sin cancels).  The rounding to the 16-bit precision is done by the fp64 adder
+// (add and subtract a power of two chosen from the value's exponent), after which the
+// narrowing conversions are exact.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -20,19 +25,44 @@ namespace {
 constexpr int kRopeThreads = 128;
 
 template <bool kBf16>
-__device__ __forceinline__ float load16(uint32_t word, int hi) {
+__device__ __forceinline__ double load16(uint32_t word, int hi) {
     const uint16_t h = hi ? (uint16_t)(word >> 16) : (uint16_t)(word & 0xFFFFu);
-    if (kBf16) return __uint_as_float((uint32_t)h << 16);
-    return __half2float(__ushort_as_half(h));
+    if (kBf16) return (double)__uint_as_float((uint32_t)h << 16);
+    return (double)__half2float(__ushort_as_half(h));
+}
+
+// fp64 -> bit pattern of the nearest bf16 / fp16 value (ties to even), in one rounding.
+// With E the exponent of v, adding and subtracting 2^(E + 53 - p) (same sign as v) leaves v
+// rounded to p significant bits by the adder; E is clamped at the type's smallest normal
+// exponent so that subnormal results keep the subnormal spacing.  The rounded value is exact
+// in fp32 and in the 16-bit type.
+template <bool kBf16>
+__device__ __forceinline__ uint32_t round16(double v) {
+    constexpr int p = kBf16 ? 8 : 11, emin = kBf16 ? -126 : -14;
+    const int hi = __double2hiint(v);
+    const int e = max(hi & 0x7FF00000, (emin + 1023) << 20);
+    double r = v;
+    if (e < 0x7FF00000) {  // finite
+        const double big = __hiloint2double((hi & (int)0x80000000) | (e + ((53 - p) << 20)), 0);
+        r = __dsub_rn(__dadd_rn(v, big), big);
+    }
+    const float f = __double2float_rn(r);  // exact (or inf / nan)
+    uint32_t bits;
+    if (kBf16)
+        bits = __float_as_uint(f) >> 16;
+    else
+        bits = (uint32_t)__half_as_ushort(__float2half_rn(f));
+    return (bits & 0x7FFFu) | (((uint32_t)hi >> 16) & 0x8000u);  // keeps the sign of a zero
 }
 template <bool kBf16>
-__device__ __forceinline__ uint32_t pack16(float lo, float hi) {
-    if (kBf16) {
-        return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) |
-               ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
-    }
-    return (uint32_t)__half_as_ushort(__float2half_rn(lo)) |
-           ((uint32_t)__half_as_ushort(__float2half_rn(hi)) << 16);
+__device__ __forceinline__ uint32_t pack16(double lo, double hi) {
+    return round16<kBf16>(lo) | (round16<kBf16>(hi) << 16);
+}
+// one pair turned by the angle whose cosine and sine are c and s: each product and each sum is
+// a separately rounded fp64 operation
+__device__ __forceinline__ void turn(double x, double y, double c, double s, double& xo, double& yo) {
+    xo = __dsub_rn(__dmul_rn(x, c), __dmul_rn(y, s));
+    yo = __dadd_rn(__dmul_rn(x, s), __dmul_rn(y, c));
 }
 
 template <bool kBf16>
@@ -47,15 +77,15 @@ __global__ void __launch_bounds__(kRopeThreads) rerotate_kernel(const RopeParams
     const int delta = j - p.keep_idx[(size_t)s * p.keep_stride + j];
     if (delta == 0) return;  // the row did not move
 
-    float cs[8], sn[8];
+    double cs[8], sn[8];
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
         const int i = 8 * u + q;
         const double theta = exp2(-(double)(2 * i) / (double)p.head_dim * p.log2_base);
         double sv, cv;
         sincos((double)delta * theta, &sv, &cv);
-        cs[q] = (float)cv;
-        sn[q] = (float)sv;
+        cs[q] = cv;
+        sn[q] = sv;
     }
     const size_t row_bytes = (size_t)p.head_dim * 2;
     const int pl0 = blockIdx.z * p.planes_per_group;
@@ -71,25 +101,22 @@ __global__ void __launch_bounds__(kRopeThreads) rerotate_kernel(const RopeParams
         if (p.layout == SIRLLM_ROPE_HALF) {  // a holds x of pairs 8u..8u+7, b holds their y
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                float x[2], y[2];
+                double x[2], y[2];
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const float xv = load16<kBf16>(wa[q], h), yv = load16<kBf16>(wb[q], h);
-                    x[h] = fmaf(xv, cs[2 * q + h], -(yv * sn[2 * q + h]));
-                    y[h] = fmaf(xv, sn[2 * q + h], yv * cs[2 * q + h]);
-                }
+                for (int h = 0; h < 2; ++h)
+                    turn(load16<kBf16>(wa[q], h), load16<kBf16>(wb[q], h), cs[2 * q + h],
+                         sn[2 * q + h], x[h], y[h]);
                 oa[q] = pack16<kBf16>(x[0], x[1]);
                 ob[q] = pack16<kBf16>(y[0], y[1]);
             }
         } else {  // every 32-bit word is one pair (x, y): a = pairs 8u..8u+3, b = 8u+4..8u+7
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                float xv = load16<kBf16>(wa[q], 0), yv = load16<kBf16>(wa[q], 1);
-                oa[q] = pack16<kBf16>(fmaf(xv, cs[q], -(yv * sn[q])), fmaf(xv, sn[q], yv * cs[q]));
-                xv = load16<kBf16>(wb[q], 0);
-                yv = load16<kBf16>(wb[q], 1);
-                ob[q] = pack16<kBf16>(fmaf(xv, cs[4 + q], -(yv * sn[4 + q])),
-                                      fmaf(xv, sn[4 + q], yv * cs[4 + q]));
+                double xo, yo;
+                turn(load16<kBf16>(wa[q], 0), load16<kBf16>(wa[q], 1), cs[q], sn[q], xo, yo);
+                oa[q] = pack16<kBf16>(xo, yo);
+                turn(load16<kBf16>(wb[q], 0), load16<kBf16>(wb[q], 1), cs[4 + q], sn[4 + q], xo, yo);
+                ob[q] = pack16<kBf16>(xo, yo);
             }
         }
         *pa = make_uint4(oa[0], oa[1], oa[2], oa[3]);

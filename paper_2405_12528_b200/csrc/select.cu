@@ -23,10 +23,10 @@ namespace {
 constexpr int kSelectThreads = 1024;
 constexpr int kRadixBits = 11;
 constexpr int kRadixBins = 1 << kRadixBits;
-constexpr int kListMax = 256;  // keys ranked directly once the radix bin holds no more
+constexpr int kListMax = 256;  // keys ranked directly once a radix bin holds no more
 
 struct BlockScratch {
-    int warp_sum[32];
+    uint32_t warp_sum[32];
     uint32_t red_min[32];
     uint32_t red_max[32];
     int bin;
@@ -38,21 +38,21 @@ struct BlockScratch {
     int first_evicted;
 };
 
-// inclusive prefix sum over the 1024 threads of the block
-__device__ __forceinline__ int block_inclusive_scan(int v, int* warp_sum) {
+// inclusive prefix sum over the 1024 threads of the block (unsigned: wraps, never overflows)
+__device__ __forceinline__ uint32_t block_inclusive_scan_u32(uint32_t v, uint32_t* warp_sum) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        int n = __shfl_up_sync(0xFFFFFFFFu, v, o);
+        const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, v, o);
         if (lane >= o) v += n;
     }
     if (lane == 31) warp_sum[wid] = v;
     __syncthreads();
     if (wid == 0) {
-        int w = warp_sum[lane];
+        uint32_t w = warp_sum[lane];
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            int n = __shfl_up_sync(0xFFFFFFFFu, w, o);
+            const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, w, o);
             if (lane >= o) w += n;
         }
         warp_sum[lane] = w;
@@ -60,6 +60,9 @@ __device__ __forceinline__ int block_inclusive_scan(int v, int* warp_sum) {
     __syncthreads();
     if (wid > 0) v += warp_sum[wid - 1];
     return v;
+}
+__device__ __forceinline__ int block_inclusive_scan(int v, uint32_t* warp_sum) {
+    return (int)block_inclusive_scan_u32((uint32_t)v, warp_sum);
 }
 
 // kStage: the keep list is assembled in shared memory and written out coalesced (the host
@@ -79,18 +82,25 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     float* scores = p.scores + (size_t)s * cap;
     int32_t* keep = p.keep_idx + (size_t)s * p.threshold;
     grid_launch_dependents();
-    grid_dependency_wait();  // the scorer's appended scores
-    if (blockIdx.x == 0 && tid == 0) *p.epoch += 1;  // a new compaction follows
-
+    // In the fused round this grid may become resident while the scorer is still draining
+    // (programmatic dependent launch).  Everything up to grid_dependency_wait() uses only
+    // what the scorer does not produce - the lengths, the decay ratio and the l0 scores held
+    // from earlier rounds - so it overlaps the scorer's tail; only the round's T new scores
+    // are folded in after the wait.
     const int l0 = p.live_len[s];
     const float eta = p.decay[s];  // fetched together with the lengths: one round trip
     int T = 0;
-    if (p.score_new) {  // the scorer has appended T raw scores behind slot l0
+    if (p.score_new) {  // the scorer appends T raw scores behind slot l0
         T = p.n_new ? p.n_new[s] : p.max_new;
         T = max(0, min(T, p.max_new));
     }
     if (l0 < 0 || l0 > cap - T) {  // the round does not fit: leave the stream alone
+        grid_dependency_wait();
         if (tid == 0) {
+            if (blockIdx.x == 0) {
+                *p.epoch += 1;
+                *p.ticket = 0ull;
+            }
             atomicOr(p.status, SIRLLM_STATUS_OVERFLOW);
             const int n = max(0, min(l0, min(cap, p.threshold)));
             p.n_keep[s] = n;
@@ -108,28 +118,37 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     constexpr int kLoadBatch = 16;
     const int lo = p.n_sink, hi = l - p.n_recent;
     uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;  // over the middle slots' keys (for S4)
-    for (int base = 0; base < l; base += kLoadBatch * kSelectThreads) {
-        float x[kLoadBatch];
+    auto decay_range = [&](int begin, int end) {
+        for (int base = begin; base < end; base += kLoadBatch * kSelectThreads) {
+            float x[kLoadBatch];
 #pragma unroll
-        for (int q = 0; q < kLoadBatch; ++q) {
-            const int i = base + q * kSelectThreads + tid;
-            x[q] = i < l ? scores[i] : 0.f;
-        }
+            for (int q = 0; q < kLoadBatch; ++q) {
+                const int i = base + q * kSelectThreads + tid;
+                x[q] = i < end ? scores[i] : 0.f;
+            }
 #pragma unroll
-        for (int q = 0; q < kLoadBatch; ++q) {
-            const int i = base + q * kSelectThreads + tid;
-            if (i < l) {
-                const float v = __fmul_rn(x[q], eta);
-                vals[i] = __float_as_uint(v);
-                if (write_now) scores[i] = v;
-                if (i >= lo && i < hi) {
-                    const uint32_t key = order_key(__float_as_uint(v));
-                    kmin = min(kmin, key);
-                    kmax = max(kmax, key);
+            for (int q = 0; q < kLoadBatch; ++q) {
+                const int i = base + q * kSelectThreads + tid;
+                if (i < end) {
+                    const float v = __fmul_rn(x[q], eta);
+                    vals[i] = __float_as_uint(v);
+                    if (write_now) scores[i] = v;
+                    if (i >= lo && i < hi) {
+                        const uint32_t key = order_key(__float_as_uint(v));
+                        kmin = min(kmin, key);
+                        kmax = max(kmax, key);
+                    }
                 }
             }
         }
+    };
+    decay_range(0, l0);      // the scores of earlier rounds
+    grid_dependency_wait();  // the scorer's appended scores are complete and visible
+    if (blockIdx.x == 0 && tid == 0) {  // a new compaction follows
+        *p.epoch += 1;
+        *p.ticket = 0ull;
     }
+    decay_range(l0, l);      // this round's scores
     if (!evict) {  // ---- nothing to evict: identity keep list --------------------------
         for (int i = tid; i < l; i += kSelectThreads) keep[i] = i;
         if (tid == 0) {
@@ -258,11 +277,12 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
         }
     }
     if (tid == 0) sh.first_evicted = l;
-    // both counts are at most 49152 < 2^16: one packed scan
-    const int packed = n_sure | (n_eq << 16);
-    const int before = block_inclusive_scan(packed, sh.warp_sum) - packed;
-    int eq_before = (int)((uint32_t)before >> 16);
-    int pos = (before & 0xFFFF) + min(eq_before, r);
+    // both counts are at most 49152 < 2^16: one scan of the two packed into an unsigned word
+    // (the scan adds ints; the sums are taken modulo 2^32, which is exact for unsigned fields)
+    const uint32_t packed = (uint32_t)n_sure | ((uint32_t)n_eq << 16);
+    const uint32_t before = block_inclusive_scan_u32(packed, sh.warp_sum) - packed;
+    int eq_before = (int)(before >> 16);
+    int pos = (int)(before & 0xFFFFu) + min(eq_before, r);
     int my_first_evicted = l;
     for (int i = i0; i < i1; i += 4) {
         const uint4 q = *reinterpret_cast<const uint4*>(vals + i);
