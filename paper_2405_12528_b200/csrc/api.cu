@@ -45,8 +45,12 @@ WorkspaceLayout workspace_layout(const sirllm_config& c) {
     L.n_part = (int32_t)((nvec + per_cta - 1) / per_cta);
     if (L.n_part < 1) L.n_part = 1;
     size_t off = 256;
-    L.plane_flags_off = off;
-    off = align_up(off + (size_t)2 * c.n_streams * c.n_layers * c.n_kv_heads * 4, 256);
+    L.plane_progress_off = off;
+    {
+        const size_t planes = (size_t)2 * c.n_streams * c.n_layers * c.n_kv_heads;
+        const size_t chained = planes < (size_t)kChainPlanesMax ? planes : (size_t)kChainPlanesMax;
+        off = align_up(off + chained * kMaxSplit * sizeof(unsigned long long), 256);
+    }
     L.first_moved_off = off;
     off = align_up(off + (size_t)c.n_streams * 4, 256);
     L.n_keep_off = off;
@@ -219,7 +223,7 @@ static int compact_params(const sirllm_config& c, const WorkspaceLayout& L, cons
     p.status = (int32_t*)ws;
     p.epoch = (int32_t*)ws + 1;
     p.ticket = (unsigned long long*)ws + 1;
-    p.plane_flags = (int32_t*)((char*)ws + L.plane_flags_off);
+    p.plane_progress = (unsigned long long*)((char*)ws + L.plane_progress_off);
     p.planes_per_stream = c.n_layers * c.n_kv_heads;
     p.planes_per_tensor = (int64_t)c.n_streams * p.planes_per_stream;
     p.capacity = c.capacity;
@@ -537,8 +541,9 @@ int sirllm_selftest_bounded_wait(const sirllm_config* cfg, void* ws, uint32_t po
     if (misaligned(ws, 256)) return SIRLLM_ERR_ALIGN;
     if (polls > (1u << 20)) return SIRLLM_ERR_BAD_CONFIG;  // keep the self-test short
     const WorkspaceLayout L = workspace_layout(*cfg);
-    cudaError_t e = launch_bounded_wait_selftest((int32_t*)((char*)ws + L.plane_flags_off), polls,
-                                                 (int32_t*)ws, (cudaStream_t)cuda_stream);
+    cudaError_t e = launch_bounded_wait_selftest(
+        (unsigned long long*)((char*)ws + L.plane_progress_off), (const int32_t*)((char*)ws + L.keep_off),
+        polls, (int32_t*)ws, (cudaStream_t)cuda_stream);
     return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "bounded_wait_selftest");
 }
 

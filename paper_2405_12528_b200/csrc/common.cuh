@@ -11,7 +11,8 @@ namespace sirllm {
 // ---- workspace layout (device memory owned by the caller) -------------------------------
 //   [0, 256)                              header: int32 status word, int32 compaction epoch,
 //                                         uint64 ticket counter of the KV gather's work units
-//   plane_flags[2*n_streams*planes]       progress of a plane split across several workers
+//   plane_progress[planes][kMaxSplit]     uint64 progress word per plane and segment, for the
+//                                         planes (at most kChainPlanesMax) that are cut into segments
 //   first_moved[n_streams]                first slot whose row changes place when compacting
 //   n_keep_fallback[n_streams]            used when the caller passes no n_keep
 //   keep_fallback[n_streams][threshold]   used when the caller passes no keep_idx
@@ -19,7 +20,7 @@ namespace sirllm {
 //   tickets[n_streams*max_new]            arrivals per logits row (the last CTA finishes the row)
 //   partials[n_streams*max_new][n_part]   (scaled max, sum) pair per CTA of a multi-CTA row
 struct WorkspaceLayout {
-    size_t plane_flags_off;
+    size_t plane_progress_off;
     size_t first_moved_off;
     size_t n_keep_off;
     size_t keep_off;
@@ -31,6 +32,8 @@ struct WorkspaceLayout {
     int32_t n_part;  // CTAs (kScoreCtaVecs vectors each) per logits row
 };
 
+constexpr int kMaxSplit = 32;           // segments a plane's moved rows may be cut into (one per lane)
+constexpr int kChainPlanesMax = 8192;   // with more K and V planes than this, planes are not cut
 constexpr int kScoreCtaVecs = 4096;  // 16-byte vectors of one logits row per CTA: 64 KB, shared
                                      // by 4 warps (16 KB each) or, in small grids, 8 or 16
 
@@ -113,7 +116,7 @@ struct CompactParams {
     int32_t* status;
     int32_t* epoch;        // bumped once per compaction by the kernel that precedes it
     unsigned long long* ticket;  // next work unit to hand out; zeroed by the same kernel
-    int32_t* plane_flags;  // [tensors * planes_per_tensor]
+    unsigned long long* plane_progress;  // [min(planes, kChainPlanesMax)][kMaxSplit]
     int64_t planes_per_tensor;  // n_streams * n_layers * n_kv_heads
     int32_t planes_per_stream;
     int32_t capacity, keep_stride, row_bytes;
@@ -131,8 +134,8 @@ cudaError_t launch_rerotate(const RopeParams& p, int n_streams, bool bf16, cudaS
 cudaError_t launch_compact_plan(const CompactParams& p, int n_streams, int32_t* first_moved,
                                 cudaStream_t st);
 cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap);
-cudaError_t launch_bounded_wait_selftest(int32_t* flag, uint32_t limit, int32_t* status,
-                                         cudaStream_t st);
+cudaError_t launch_bounded_wait_selftest(unsigned long long* prog, const int32_t* keep, uint32_t limit,
+                                         int32_t* status, cudaStream_t st);
 
 // ---- small device helpers ----------------------------------------------------------------
 #ifdef __CUDACC__
@@ -168,8 +171,11 @@ __device__ __forceinline__ void mbar_init_fence() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
+// The one arrival of a stage's phase plus the bytes its bulk loads will deliver.  Relaxed: the
+// arrival publishes nothing (the stage record written before it is read back by the same warp
+// after a __syncwarp), so it need not wait for earlier shared-memory stores.
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+    asm volatile("mbarrier.arrive.expect_tx.relaxed.cta.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
                  "r"(bytes)
                  : "memory");
 }
@@ -217,25 +223,20 @@ __device__ __forceinline__ void bulk_wait_all() {
 }
 // polls before a device-side wait gives up (a healthy wait ends within microseconds for an
 // mbarrier and within one kernel duration for a progress word; these limits are seconds)
-constexpr uint32_t kSpinLimit = 1u << 22;      // global-memory progress words
+constexpr uint32_t kSpinLimit = 1u << 22;      // global-memory progress words (>= 200 ns a poll)
 constexpr uint32_t kMbarSpinLimit = 1u << 20;  // mbarrier phases (each poll may itself suspend)
 
-// Progress words in global memory (release / acquire at GPU scope) and the bounded wait on them.
-__device__ __forceinline__ uint32_t ld_acquire(const int32_t* p) {
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+// Progress words in global memory, GPU scope.
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_release(int32_t* p, uint32_t v) {
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-// false if *flag did not become `want` within `limit` polls
-__device__ __forceinline__ bool wait_progress_word(const int32_t* flag, uint32_t want, uint32_t limit) {
-    uint32_t spins = 0;
-    while (ld_acquire(flag) != want) {
-        if (++spins > limit) return false;
-    }
-    return true;
+// A progress word carries no data besides itself (what it announces - bulk loads that have
+// landed - completed before the announcing thread saw their mbarrier flip), so it is written
+// relaxed: a release store would first wait for every load the thread still has in flight.
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
 // Order-preserving map from fp32 bit patterns to unsigned integers: a larger key is a

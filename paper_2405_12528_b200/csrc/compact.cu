@@ -18,14 +18,23 @@
 // To fill all SMs evenly, the moved rows of a plane are cut into `split` segments that
 // different workers take.  Work units (plane, segment) are numbered segment-major, so a
 // plane's earlier segments come long before its later ones, and are handed out in that order
-// through one ticket counter in the workspace: a worker that is ready draws the next number.
-// A segment may store only after every earlier segment of its plane has landed all its loads;
-// that is tracked by one progress word per plane (epoch * 64 + finished segments) written
-// with release and polled with acquire, with an iteration limit.  A worker only ever waits
-// for a unit with a smaller number than its own, and every smaller number was drawn by a
-// worker that is running (it drew the number itself), so by induction the waits end whatever
-// number of CTAs the device keeps resident at once; the hand-out also evens out SMs that run
-// at different speeds.
+// through one ticket counter in the workspace: a worker that is about to run dry draws the
+// next number.  That evens out SMs that run at different speeds.
+//
+// A segment's stores overwrite rows that may still be the sources of EARLIER segments of the
+// plane (never of later ones: keep[j] >= j).  Every segment therefore publishes how many of
+// its chunks have landed in shared memory (one 64-bit progress word per plane and segment:
+// compaction epoch | chunk count).  Before a chunk with destination
+// rows [d0, d1) is stored, the worker makes sure that every destination row j in front of
+// its segment whose source keep[j] lies below d1 has landed: it reads the earlier segments'
+// progress words (one per lane, acquire), finds J = the number of leading rows of the plane
+// known to have landed, and may then store anything below keep[J] (all of the plane once the
+// earlier segments are complete).  The bound is remembered, so a segment polls again only
+// when it outruns it; with rows moving by many slots, the rows a segment overwrites were read
+// long before.  The wait has an iteration limit.  A worker only ever waits for units with a
+// smaller number than its own, and every smaller number was drawn by a worker that is
+// running (it drew the number itself), so by induction the waits end whatever number of CTAs
+// the device keeps resident at once.
 #include "common.cuh"
 
 namespace sirllm {
@@ -35,37 +44,109 @@ namespace {
 constexpr int kChunkRows = 32;  // rows per chunk = one per lane
 constexpr int kStoreSlack = 1;  // bulk stores that may still be reading shared memory
 constexpr int kMaxStages = 12;
-constexpr int kMaxSplit = 32;
-constexpr int kIdxAhead = 4;  // chunks whose source indices are fetched ahead
-constexpr int kMaxWorkers = 4;  // worker warps per CTA
+constexpr int kIdxAhead = 4;     // chunks whose source indices are fetched ahead
+constexpr int kMaxWorkers = 4;   // worker warps per CTA
+constexpr int kPublishEvery = 4; // chunks between two updates of a segment's progress word
+constexpr int kNoBound = 0x7FFFFFFF;
 
+// What the store of a chunk needs to know about the chunk ...
 struct StageInfo {
-    char* dst;           // destination of the chunk held by the stage
-    int32_t* flag;       // progress word of the chunk's plane
+    char* dst;         // destination of the chunk held by the stage
     uint32_t bytes;
-    uint32_t wait_val;   // != 0: the store must wait until *flag == wait_val
-    uint32_t signal_val; // != 0: once the chunk's loads have landed set *flag = signal_val
-    uint32_t pad;
+    int32_t d_end;     // one past the chunk's last destination row; 0: no earlier segment to mind
+    uint32_t publish;  // != 0: chunks of this segment that have landed once this one has
+    uint32_t unit;     // running number of the worker's work unit the chunk belongs to
+};
+// ... and about the work unit (plane, segment) it belongs to; written once per unit.
+struct UnitInfo {
+    const int32_t* keep;       // keep list of the unit's stream
+    unsigned long long* prog;  // progress words of the unit's plane, one per segment
+    int32_t seg;               // segment of the plane
+    int32_t first;             // first moved row of the stream
+    int32_t seg_rows;          // rows per (full) segment
+    int32_t n;                 // rows kept in the stream
 };
 
-// Lane 0 waits for the loads of chunk c, honours the plane's progress word and stores the
-// chunk.  Returns false (to all lanes) if a wait ran out.
-__device__ __forceinline__ bool store_chunk(uint64_t* full, StageInfo* info, char* buf, int64_t c,
-                                            int stages, uint32_t stage_bytes, int lane) {
-    bool ok = true;
+// What a worker knows about the earlier segments of the unit it is storing.
+struct SafeBound {
+    uint32_t unit = 0xFFFFFFFFu;
+    int32_t below = 0;  // destination rows below this one may be stored
+};
+
+// Before a chunk of a later segment is stored: wait (whole warp, at most `limit` polls) until
+// no earlier segment of the plane still has to read the rows below d_end.
+__device__ __forceinline__ bool wait_for_earlier_segments(const UnitInfo& ui, int32_t d_end, uint32_t unit,
+                                                          uint32_t epoch, SafeBound& safe, int lane,
+                                                          uint32_t limit) {
+    if (safe.unit != unit) {
+        safe.unit = unit;
+        safe.below = 0;
+    }
+    uint32_t polls = 0;
+    while (d_end > safe.below) {
+        // lane g looks at segment g < seg: has it landed all its chunks, if not how many
+        const int total = (ui.n - ui.first + kChunkRows - 1) / kChunkRows;
+        const int per_seg = ui.seg_rows / kChunkRows;
+        int landed = 0;
+        bool done = true;
+        if (lane < ui.seg) {
+            const unsigned long long v = ld_acquire_u64(ui.prog + lane);
+            landed = (v >> 32) == (unsigned long long)epoch ? (int)(uint32_t)v : 0;
+            done = landed >= min(per_seg, total - lane * per_seg);
+        }
+        const uint32_t open = __ballot_sync(0xFFFFFFFFu, !done);
+        if (open == 0) {
+            safe.below = kNoBound;  // everything in front of the segment has landed
+        } else {
+            // rows in front of J = first row not known to have landed; sources below keep[J]
+            // all belong to rows in front of J
+            const int g = __ffs(open) - 1;
+            const int rows_in = __shfl_sync(0xFFFFFFFFu, landed, g) * kChunkRows;
+            int bound = 0;
+            if (lane == 0) bound = ui.keep[ui.first + g * ui.seg_rows + rows_in];
+            safe.below = __shfl_sync(0xFFFFFFFFu, bound, 0);
+        }
+        if (d_end <= safe.below) break;
+        if (++polls > limit) return false;
+        __nanosleep(200);
+    }
+    return true;
+}
+
+// Lane 0 waits for the loads of chunk c and publishes the segment's progress; for a chunk of a
+// later segment the warp makes sure no earlier segment still needs the rows the chunk
+// overwrites; lane 0 stores the chunk.  Returns false (to all lanes) if a wait ran out.
+__device__ __forceinline__ bool store_chunk(uint64_t* full, const StageInfo* info, const UnitInfo* units,
+                                            char* buf, int64_t c, int stages, uint32_t stage_bytes,
+                                            int lane, uint32_t epoch, SafeBound& safe) {
+    const int stage = (int)(c % stages);
+    const StageInfo* si = &info[stage];
+    int ok = 1;
     if (lane == 0) {
-        const int stage = (int)(c % stages);
-        const uint32_t parity = (uint32_t)((c / stages) & 1);
-        ok = mbar_wait_bounded(&full[stage], parity, kMbarSpinLimit);
-        const StageInfo si = info[stage];
-        if (ok && si.wait_val != 0) ok = wait_progress_word(si.flag, si.wait_val, kSpinLimit);
-        if (ok) {
-            if (si.signal_val != 0) st_release(si.flag, si.signal_val);
-            bulk_store(si.dst, buf + (size_t)stage * stage_bytes, si.bytes);
-            bulk_commit();
+        ok = mbar_wait_bounded(&full[stage], (uint32_t)((c / stages) & 1), kMbarSpinLimit);
+        if (ok && si->publish != 0) {
+            const UnitInfo* ui = &units[si->unit % kMaxStages];
+            st_relaxed_u64(ui->prog + ui->seg, ((unsigned long long)epoch << 32) | si->publish);
         }
     }
-    return __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+    const int32_t d_end = si->d_end;  // the same word for every lane
+    if (d_end != 0) {
+        ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+        if (ok) {
+            const uint32_t unit = si->unit;
+            ok = wait_for_earlier_segments(units[unit % kMaxStages], d_end, unit, epoch, safe, lane, kSpinLimit);
+        }
+    }
+    if (lane == 0 && ok) {
+        bulk_store(si->dst, buf + (size_t)stage * stage_bytes, si->bytes);
+        bulk_commit();
+    }
+    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+}
+
+__host__ __device__ inline size_t header_bytes(int n_workers) {
+    const size_t h = (size_t)n_workers * kMaxStages * (8 + sizeof(StageInfo) + sizeof(UnitInfo));
+    return (h + 127) & ~(size_t)127;
 }
 
 __global__ void __launch_bounds__(kMaxWorkers * 32, 1)
@@ -75,12 +156,15 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
     const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t stage_bytes = (uint32_t)kChunkRows * (uint32_t)p.row_bytes;
 
-    // shared memory: [workers][kMaxStages] mbarriers and stage records, then the rings
+    // shared memory: [workers][kMaxStages] mbarriers, stage records and unit records (chunks
+    // in flight belong to at most `stages` units), then the rings
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw) + wid * kMaxStages;
     StageInfo* info =
         reinterpret_cast<StageInfo*>(smem_raw + (size_t)n_workers * kMaxStages * 8) + wid * kMaxStages;
-    size_t header = (size_t)n_workers * kMaxStages * (8 + sizeof(StageInfo));
-    header = (header + 127) & ~(size_t)127;
+    UnitInfo* units = reinterpret_cast<UnitInfo*>(smem_raw + (size_t)n_workers * kMaxStages *
+                                                                 (8 + sizeof(StageInfo))) +
+                      wid * kMaxStages;
+    size_t header = header_bytes(n_workers);
     char* buf = reinterpret_cast<char*>(smem_raw) + header + (size_t)wid * stages * stage_bytes;
 
     if (lane == 0) {
@@ -88,22 +172,27 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
         mbar_init_fence();
     }
     __syncwarp();
-    grid_dependency_wait();  // the keep lists (and the epoch) of the preceding kernel
+    grid_dependency_wait();  // the keep lists, the epoch and the ticket counter of the preceding kernel
 
-    const uint32_t epoch_base = ((uint32_t)*p.epoch << 6) | 0x80000000u;  // never 0
+    const uint32_t epoch = (uint32_t)*p.epoch;
     const int lead = stages - 1 - kStoreSlack;  // chunks whose loads run ahead of the stores
     const int64_t n_units = (int64_t)units_base * split;
     int64_t it = 0;      // chunks whose loads were issued
     int64_t stored = 0;  // chunks whose store was issued
+    uint32_t unit_no = 0;
     bool alive = true;
+    SafeBound safe;
 
-    // the next unit's number is drawn while the current unit is being moved
-    unsigned long long drawn = 0;
+    unsigned long long drawn = 0;  // lane 0: the number of the next unit
     if (lane == 0) drawn = atomicAdd(p.ticket, 1ull);
     while (alive) {
         const int64_t u = (int64_t)__shfl_sync(0xFFFFFFFFu, drawn, 0);
         if (u >= n_units) break;
-        if (lane == 0) drawn = atomicAdd(p.ticket, 1ull);
+        bool need_draw = true;  // the next number is drawn towards the end of this unit
+        auto draw = [&]() {
+            if (need_draw && lane == 0) drawn = atomicAdd(p.ticket, 1ull);
+            need_draw = false;
+        };
         const int h = (int)(u / units_base);  // segment of the plane's moved rows
         const int r = (int)(u - (int64_t)h * units_base);
         const int tensor = (int)(r / p.planes_per_tensor);
@@ -111,13 +200,15 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
         const int s = (int)(plane / p.planes_per_stream);
         const int n = min(max(p.n_keep[s], 0), p.keep_stride);
         int f = p.first_moved[s];
-        if (f < 0) continue;  // keep list rejected
-        if (!p.in_place) f = 0;
-        if (f >= n) continue;
-        const int total_chunks = (n - f + kChunkRows - 1) / kChunkRows;
-        const int per_seg = (total_chunks + split - 1) / split;
+        if (!p.in_place && f >= 0) f = 0;
+        const int total_chunks = f >= 0 && f < n ? (n - f + kChunkRows - 1) / kChunkRows : 0;
+        const int per_seg = max((total_chunks + split - 1) / split, 1);
         const int n_seg = (total_chunks + per_seg - 1) / per_seg;  // non-empty segments
-        if (h >= n_seg) continue;
+        if (h >= n_seg) {  // keep list rejected, nothing moves, or fewer segments than `split`
+            draw();
+            continue;
+        }
+        ++unit_no;  // counts the units that put chunks into the ring
         const int c_begin = h * per_seg, c_end = min(total_chunks, c_begin + per_seg);
         const int j_begin = f + c_begin * kChunkRows, j_end = min(n, f + c_end * kChunkRows);
 
@@ -125,6 +216,16 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
         char* dst = (tensor ? p.dst[1] : p.dst[0]) + (size_t)plane * p.capacity * p.row_bytes;
         const int32_t* keep = p.keep_idx + (size_t)s * p.keep_stride;
         const bool chained = p.in_place && n_seg > 1;
+        if (chained && lane == 0) {
+            UnitInfo ui;
+            ui.keep = keep;
+            ui.prog = p.plane_progress + (size_t)r * kMaxSplit;
+            ui.seg = h;
+            ui.first = f;
+            ui.seg_rows = per_seg * kChunkRows;
+            ui.n = n;
+            units[unit_no % kMaxStages] = ui;
+        }
 
         // source rows of the next kIdxAhead chunks, one per lane and chunk, fetched a whole
         // group ahead so that the index loads never sit on the critical path
@@ -135,6 +236,7 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
             kq[q] = j < j_end ? keep[j] : -2;
         }
         for (int jg = j_begin; jg < j_end && alive; jg += kIdxAhead * kChunkRows) {
+            if (jg + 2 * kIdxAhead * kChunkRows >= j_end) draw();
             int kn[kIdxAhead];
 #pragma unroll
             for (int q = 0; q < kIdxAhead; ++q) {
@@ -152,13 +254,14 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
                     if (it >= stages) bulk_wait_read<kStoreSlack>();  // the stage's last store has left
                     StageInfo si;
                     si.dst = dst + (size_t)j0 * p.row_bytes;
-                    si.flag = p.plane_flags + r;
                     si.bytes = (uint32_t)nrows * p.row_bytes;
-                    si.wait_val = (chained && h > 0 && j0 == j_begin) ? epoch_base + h : 0u;
-                    si.signal_val = (chained && h + 1 < n_seg && j0 + kChunkRows >= j_end)
-                                        ? epoch_base + h + 1
-                                        : 0u;
-                    si.pad = 0;
+                    si.d_end = (chained && h > 0) ? j0 + nrows : 0;
+                    si.unit = unit_no;
+                    const int done = (j0 - j_begin) / kChunkRows + 1;  // chunks of the segment so far
+                    si.publish = (chained && h + 1 < n_seg &&
+                                  (done % kPublishEvery == 0 || j0 + kChunkRows >= j_end))
+                                     ? (uint32_t)done
+                                     : 0u;
                     info[stage] = si;
                     mbar_expect_tx(&full[stage], si.bytes);
                 }
@@ -176,16 +279,17 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
                 }
                 ++it;
                 if (it - stored > lead) {
-                    alive = store_chunk(full, info, buf, stored, stages, stage_bytes, lane);
+                    alive = store_chunk(full, info, units, buf, stored, stages, stage_bytes, lane, epoch, safe);
                     ++stored;
                 }
             }
 #pragma unroll
             for (int q = 0; q < kIdxAhead; ++q) kq[q] = kn[q];
         }
+        draw();
     }
     while (alive && stored < it) {
-        alive = store_chunk(full, info, buf, stored, stages, stage_bytes, lane);
+        alive = store_chunk(full, info, units, buf, stored, stages, stage_bytes, lane, epoch, safe);
         ++stored;
     }
     if (lane == 0) {
@@ -232,19 +336,30 @@ __global__ void compact_plan_kernel(const CompactParams p, int32_t* __restrict__
     }
 }
 
-// Polls a progress word nobody sets, with the same bounded wait the gather uses, and reports
-// the expiry through the status word: lets a caller check the time-out path on a healthy GPU.
-__global__ void bounded_wait_selftest_kernel(int32_t* flag, uint32_t never, uint32_t limit,
-                                             int32_t* status) {
-    if (!wait_progress_word(flag, never, limit)) atomicOr(status, SIRLLM_STATUS_TIMEOUT);
+// Runs the gather's wait for earlier segments against a progress word that nothing sets (a
+// segment of an epoch no compaction reaches), so that it gives up after `limit` polls and
+// reports the expiry through the status word: lets a caller check the time-out path on a
+// healthy GPU.
+__global__ void bounded_wait_selftest_kernel(unsigned long long* prog, const int32_t* keep,
+                                             uint32_t limit, int32_t* status) {
+    UnitInfo ui;
+    ui.keep = keep;  // keep[0] is read: any valid word (rows below it count as safe)
+    ui.prog = prog;
+    ui.seg = 1;
+    ui.first = 0;
+    ui.seg_rows = kChunkRows;
+    ui.n = 2 * kChunkRows;
+    SafeBound safe;
+    // a row beyond any slot number, in an epoch no compaction reaches
+    const bool ok = wait_for_earlier_segments(ui, kNoBound - 1, 1u, 0xFFFFFFFFu, safe, threadIdx.x & 31, limit);
+    if (!ok && threadIdx.x == 0) atomicOr(status, SIRLLM_STATUS_TIMEOUT);
 }
 
 }  // namespace
 
-cudaError_t launch_bounded_wait_selftest(int32_t* flag, uint32_t limit, int32_t* status,
-                                         cudaStream_t st) {
-    // progress words always have their top bit set; 1 is a value none of them ever takes
-    bounded_wait_selftest_kernel<<<1, 1, 0, st>>>(flag, 1u, limit, status);
+cudaError_t launch_bounded_wait_selftest(unsigned long long* prog, const int32_t* keep, uint32_t limit,
+                                         int32_t* status, cudaStream_t st) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(prog, keep, limit, status);
     return cudaGetLastError();
 }
 
@@ -286,9 +401,7 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     while (stages > 4 && (size_t)workers * stages * stage_bytes > budget) --stages;
     if ((size_t)workers * stages * stage_bytes > budget) return cudaErrorInvalidValue;
     while (stages < 8 && (size_t)workers * (stages + 1) * stage_bytes <= budget) ++stages;
-    size_t header = (size_t)workers * kMaxStages * (8 + sizeof(StageInfo));
-    header = (header + 127) & ~(size_t)127;
-    const size_t smem = header + (size_t)workers * stages * stage_bytes;
+    const size_t smem = header_bytes(workers) + (size_t)workers * stages * stage_bytes;
     e = cudaFuncSetAttribute(compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
 
@@ -303,7 +416,7 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     // worker-rounds, then fewest segments
     const int64_t slots = resident * workers;
     int split = 1;
-    if (units_base < 8 * slots) {
+    if (units_base < 8 * slots && units_base <= kChainPlanesMax) {
         double best = -1.0;
         for (int h = 1; h <= kMaxSplit; ++h) {
             const int64_t units = (int64_t)units_base * h;
