@@ -139,6 +139,29 @@ int sirllm_score_pairs(const sirllm_config *cfg, const void *pairs, int32_t n_ti
                        void *ws, void *cuda_stream);
 
 /*
+ * Token Entropy under a vocabulary-parallel LM head (Section 3.2: the same e_i; the sum over
+ * the vocabulary inside its softmax splits over column ranges).  The caller holds columns
+ * [col0, col0 + n_cols) of every logits row - one rank's shard - and gets, per row,
+ *     pairs_out[row * pair_stride] = (m, s) with  sum over the range of exp(z) = s * exp(m),
+ *                                    m within rounding of the range's largest logit
+ *                                    ((0, 0) for an empty or fully masked range)
+ *     target_out[row] = z[row][token_ids[row]] if that column lies in the range, else 0
+ * Ranks exchange these few bytes per row (all-gather of the pairs, sum of the targets) and
+ * finish with sirllm_score_pairs, n_tiles = number of ranks; cfg->vocab stays the FULL
+ * vocabulary (token ids are checked against it there).  Rows and streams as in sirllm_score.
+ *   logits_slice      [n_streams*max_new rows] of n_cols elements, slice_row_stride apart
+ *                     (may be NULL when n_cols is 0: a rank that owns no column)
+ *   pairs_out         float[2] x [rows * pair_stride], 8-byte aligned; pair_stride >= 1 lets a
+ *                     rank write straight into its column of a [rows][ranks] array
+ *   target_out        fp32 [rows]
+ * Rows at or beyond n_new[s] are left untouched.
+ */
+int sirllm_score_partial(const sirllm_config *cfg, const void *logits_slice, int64_t col0,
+                         int64_t n_cols, int64_t slice_row_stride, const int32_t *token_ids,
+                         const int32_t *n_new, void *pairs_out, int64_t pair_stride,
+                         float *target_out, void *ws, void *cuda_stream);
+
+/*
  * sirllm_score for callers that cannot allocate device memory.  (The paper has no
  * counterpart; this is a packaging variant of the same kernel.)
  *

@@ -43,6 +43,8 @@ def _bind(path: str):
         L.oracle_score.argtypes = [vp, ctypes.c_int, i64, i64, i64, vp, vp]
         L.oracle_score_pairs.restype = ctypes.c_int
         L.oracle_score_pairs.argtypes = [vp, i64, i64, i64, vp, vp, i64, vp]
+        L.oracle_range_pair.restype = None
+        L.oracle_range_pair.argtypes = [vp, ctypes.c_int, i64, i64, i32, vp, vp]
         L.oracle_decay.restype = None
         L.oracle_decay.argtypes = [vp, i64, f32]
         L.oracle_order_key.restype = ctypes.c_uint32
@@ -136,6 +138,23 @@ def score_pairs(pairs: torch.Tensor, target_logit: torch.Tensor, ids: torch.Tens
     out = torch.empty(T, dtype=torch.float32)
     lib().oracle_score_pairs(_ptr(pairs), T, n_tiles, n_tiles, _ptr(target_logit), _ptr(ids), vocab, _ptr(out))
     return out
+
+
+def range_pairs(logits: torch.Tensor, ids: torch.Tensor, v0: int, v1: int):
+    """What one rank of a vocabulary-parallel LM head contributes for its columns ``[v0, v1)``:
+    fp32 pairs ``[T, 2]`` (max, sum exp) and the target logits ``[T]`` (0 where the token's
+    column lies outside the range)."""
+    assert logits.dim() == 2 and logits.stride(1) == 1
+    T, V = logits.shape
+    assert 0 <= v0 <= v1 <= V
+    ids = ids.to(torch.int32).contiguous()
+    pairs = torch.zeros(T, 2, dtype=torch.float32)
+    target = torch.zeros(T, dtype=torch.float32)
+    esz = logits.element_size()
+    for t in range(T):
+        lib().oracle_range_pair(logits.data_ptr() + t * logits.stride(0) * esz, _logits_dtype(logits),
+                                v0, v1, int(ids[t]), pairs.data_ptr() + 8 * t, target.data_ptr() + 4 * t)
+    return pairs, target
 
 
 def decay(E: torch.Tensor, live_len: int, eta: float) -> None:

@@ -128,6 +128,31 @@ int oracle_score_pairs(const float *pairs, int64_t T, int64_t n_tiles, int64_t p
     return n_bad;
 }
 
+/*
+ * One rank's share of a logits row under a vocabulary-parallel LM head (Section 3.2, the sum in
+ * the softmax split over column ranges): for the columns [v0, v1) of the row,
+ *     m = max of the logits,   s = sum exp(z - m)   (m = 0, s = 0 for an empty or fully masked
+ * range), both in double and rounded once to fp32; and the target logit z[id] if v0 <= id < v1,
+ * else 0.  The pairs of all ranges of a row feed oracle_entropy_from_pairs.
+ */
+void oracle_range_pair(const void *row, int dtype, int64_t v0, int64_t v1, int32_t id, float *pair,
+                       float *target)
+{
+    double m = -INFINITY;
+    for (int64_t v = v0; v < v1; ++v) {
+        double z = logit_at(row, dtype, v);
+        if (z > m)
+            m = z;
+    }
+    double s = 0.0;
+    if (m > -INFINITY)
+        for (int64_t v = v0; v < v1; ++v)
+            s += exp(logit_at(row, dtype, v) - m);
+    pair[0] = s > 0.0 ? (float)m : 0.0f;
+    pair[1] = (float)s;
+    *target = (id >= 0 && (int64_t)id >= v0 && (int64_t)id < v1) ? (float)logit_at(row, dtype, id) : 0.0f;
+}
+
 /* Memory decay (Section 3.3, E = E x eta_decay; Algorithm 1 applies it once per
  * round, after the round's scores were appended): one fp32 multiply per entry. */
 void oracle_decay(float *E, int64_t l, float eta)

@@ -24,6 +24,7 @@ POLICY_STREAM, POLICY_RANDOM, POLICY_INTERVAL = 1, 2, 3
 ROPE_HALF, ROPE_INTERLEAVED = 0, 1
 
 EXPORTS = ["sirllm_workspace_bytes", "sirllm_workspace_init", "sirllm_score", "sirllm_score_static",
+           "sirllm_score_partial",
            "sirllm_score_pairs", "sirllm_step_pairs", "sirllm_decay_select", "sirllm_keep_policy", "sirllm_rerotate_keys",
            "sirllm_compact_kv", "sirllm_step", "sirllm_step_phases", "sirllm_step_host",
            "sirllm_selftest_bounded_wait", "sirllm_status", "sirllm_strerror",
@@ -97,6 +98,9 @@ def lib():
         L.sirllm_score.argtypes = [cfgp, vp, vp, vp, vp, vp, vp]
         L.sirllm_score_static.restype = ctypes.c_int
         L.sirllm_score_static.argtypes = [cfgp, vp, vp, vp, vp, vp, vp]
+        L.sirllm_score_partial.restype = ctypes.c_int
+        L.sirllm_score_partial.argtypes = [cfgp, vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, vp, vp,
+                                           vp, ctypes.c_int64, vp, vp, vp]
         L.sirllm_score_pairs.restype = ctypes.c_int
         L.sirllm_score_pairs.argtypes = [cfgp, vp, i32, ctypes.c_int64, vp, vp, vp, vp, vp, vp]
         L.sirllm_step_pairs.restype = ctypes.c_int
@@ -328,6 +332,50 @@ def sirllm_score_static(cfg: Config, logits, token_ids, n_new, out_entropy, stat
     _call(lib().sirllm_score_static, cfg, _logits(cfg, logits),
           *_score_args(cfg, token_ids, n_new, out_entropy), _dev(status, torch.int32, "status", 1),
           _stream())
+
+
+class _SliceArg(_Arg):
+    """One rank's column range of the logits: [>= rows, n_cols], last dimension dense."""
+
+    def __init__(self, cfg, t, col0):
+        super().__init__(t, None, "logits_slice")
+        self.cfg, self.col0 = cfg, int(col0)
+
+    def check_shape(self):
+        cfg, t = self.cfg, self.t
+        if t is None:
+            raise SirllmError(ERR_NULL, "logits_slice is required")
+        if _DTYPE_CODE.get(t.dtype) != cfg.logits_dtype:
+            raise SirllmError(ERR_BAD_CONFIG, f"logits_slice dtype {t.dtype} does not match the config")
+        if t.dim() != 2 or t.shape[0] < _rows(cfg) or self.col0 < 0 or self.col0 + t.shape[1] > cfg.vocab:
+            raise SirllmError(ERR_BAD_CONFIG, f"logits_slice has shape {tuple(t.shape)} at column "
+                                              f"{self.col0}, the configuration needs [>= {_rows(cfg)}, "
+                                              f"<= {cfg.vocab - self.col0}]")
+        if t.shape[1] > 0 and t.stride(1) != 1:
+            raise SirllmError(ERR_ALIGN, "logits_slice rows must be dense")
+
+    @property
+    def row_stride(self) -> int:
+        t = self.t
+        return int(t.stride(0)) if t.shape[0] > 1 and t.shape[1] > 0 else max(int(t.shape[1]), 1)
+
+
+def sirllm_score_partial(cfg: Config, logits_slice, col0: int, token_ids, n_new, pairs_out, target_out,
+                         ws, pair_column: int = 0) -> None:
+    """One rank's share of vocabulary-parallel scoring: ``logits_slice`` holds columns
+    ``[col0, col0 + n_cols)``; ``pairs_out`` is ``[rows, n_ranks, 2]`` fp32 and this call fills
+    column ``pair_column`` of it; ``target_out`` is fp32 ``[rows]``."""
+    sl = _SliceArg(cfg, logits_slice, col0)
+    sl.check_shape()
+    pa = _PairsArg(cfg, pairs_out)
+    pa.check_shape()
+    if not 0 <= pair_column < pa.n_tiles:
+        raise SirllmError(ERR_BAD_CONFIG, f"pair_column {pair_column} outside [0, {pa.n_tiles})")
+    ids, nn, tgt = _score_args(cfg, token_ids, n_new, target_out)
+    tgt.name = "target_out"
+    pa.check_residence()
+    _call(lib().sirllm_score_partial, cfg, sl, int(col0), int(logits_slice.shape[1]), sl.row_stride,
+          ids, nn, pairs_out.data_ptr() + 8 * int(pair_column), pa.row_stride, tgt, _ws(cfg, ws), _stream())
 
 
 def sirllm_score_pairs(cfg: Config, pairs, target_logit, token_ids, n_new, out_entropy, ws) -> None:

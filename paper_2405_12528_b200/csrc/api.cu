@@ -53,6 +53,8 @@ WorkspaceLayout workspace_layout(const sirllm_config& c) {
     }
     L.first_moved_off = off;
     off = align_up(off + (size_t)c.n_streams * 4, 256);
+    L.ready_off = off;
+    off = align_up(off + (size_t)c.n_streams * 4, 256);
     L.n_keep_off = off;
     off = align_up(off + (size_t)c.n_streams * 4, 256);
     L.keep_off = off;
@@ -83,6 +85,10 @@ static ScoreParams score_params(const sirllm_config& c, const WorkspaceLayout& L
     sp.out_entropy = nullptr;
     sp.scores = nullptr;
     sp.live_len = nullptr;
+    sp.pairs_out = nullptr;
+    sp.target_out = nullptr;
+    sp.pair_stride = 0;
+    sp.col0 = 0;
     sp.capacity = c.capacity;
     sp.vocab = c.vocab;
     sp.row_stride = c.logits_row_stride;
@@ -132,6 +138,34 @@ int sirllm_score(const sirllm_config* cfg, const void* logits, const int32_t* to
     return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "score");
 }
 
+int sirllm_score_partial(const sirllm_config* cfg, const void* logits_slice, int64_t col0,
+                                    int64_t n_cols, int64_t slice_row_stride, const int32_t* token_ids,
+                                    const int32_t* n_new, void* pairs_out, int64_t pair_stride,
+                                    float* target_out, void* ws, void* cuda_stream) {
+    int rc = validate_config(cfg);
+    if (rc != SIRLLM_OK) return rc;
+    if ((!logits_slice && n_cols != 0) || !token_ids || !pairs_out || !target_out || !ws)
+        return SIRLLM_ERR_NULL;
+    if (col0 < 0 || n_cols < 0 || col0 > cfg->vocab - n_cols || slice_row_stride < n_cols || pair_stride < 1)
+        return SIRLLM_ERR_BAD_CONFIG;
+    if (misaligned(ws, 256) || misaligned(pairs_out, 8)) return SIRLLM_ERR_ALIGN;
+    if ((rc = check_logits(*cfg, logits_slice)) != SIRLLM_OK) return rc;
+    const WorkspaceLayout L = workspace_layout(*cfg);
+    ScoreParams sp = score_params(*cfg, L, logits_slice, token_ids, n_new, ws);
+    sp.pairs_out = (float2*)pairs_out;
+    sp.target_out = target_out;
+    sp.pair_stride = pair_stride;
+    sp.col0 = col0;
+    sp.vocab = n_cols;  // columns streamed; a range is never wider than the vocabulary the
+    sp.row_stride = slice_row_stride;  // workspace's per-row scratch was sized for
+    sirllm_config range = *cfg;
+    range.vocab = n_cols > 0 ? n_cols : 1;
+    range.logits_row_stride = range.vocab;
+    sp.n_part = workspace_layout(range).n_part;
+    cudaError_t e = launch_score(sp, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "score_partial");
+}
+
 static SelectParams select_params(const sirllm_config& c, const WorkspaceLayout& L, float* scores,
                                   int64_t* serial, int32_t* live_len, const float* decay,
                                   int32_t* keep_idx, int32_t* n_keep, void* ws) {
@@ -144,6 +178,7 @@ static SelectParams select_params(const sirllm_config& c, const WorkspaceLayout&
     p.keep_idx = keep_idx ? keep_idx : (int32_t*)((char*)ws + L.keep_off);
     p.n_keep = n_keep ? n_keep : (int32_t*)((char*)ws + L.n_keep_off);
     p.first_moved = (int32_t*)((char*)ws + L.first_moved_off);
+    p.ready = (int32_t*)((char*)ws + L.ready_off);
     p.status = (int32_t*)ws;
     p.epoch = (int32_t*)ws + 1;
     p.ticket = (unsigned long long*)ws + 1;
@@ -220,6 +255,7 @@ static int compact_params(const sirllm_config& c, const WorkspaceLayout& L, cons
     p.keep_idx = keep_idx;
     p.n_keep = n_keep;
     p.first_moved = (int32_t*)((char*)ws + L.first_moved_off);
+    p.ready = (int32_t*)((char*)ws + L.ready_off);
     p.status = (int32_t*)ws;
     p.epoch = (int32_t*)ws + 1;
     p.ticket = (unsigned long long*)ws + 1;

@@ -14,6 +14,7 @@ namespace sirllm {
 //   plane_progress[planes][kMaxSplit]     uint64 progress word per plane and segment, for the
 //                                         planes (at most kChainPlanesMax) that are cut into segments
 //   first_moved[n_streams]                first slot whose row changes place when compacting
+//   ready[n_streams]                      1 once a stream's keep list is complete (polled by the gather)
 //   n_keep_fallback[n_streams]            used when the caller passes no n_keep
 //   keep_fallback[n_streams][threshold]   used when the caller passes no keep_idx
 //   policy_ranks[n_streams][capacity]     synthetic scores of the comparison policies, ones[n_streams]
@@ -22,6 +23,7 @@ namespace sirllm {
 struct WorkspaceLayout {
     size_t plane_progress_off;
     size_t first_moved_off;
+    size_t ready_off;
     size_t n_keep_off;
     size_t keep_off;
     size_t tickets_off;
@@ -55,7 +57,13 @@ struct ScoreParams {
     float* out_entropy;        // [n_streams*max_new] raw scores, nullable
     float* scores;             // nullable: also append at scores[s][live_len[s] + t] (fused round)
     const int32_t* live_len;   // with `scores`
-    int64_t vocab;
+    // vocabulary-parallel mode (pairs_out != nullptr): `logits` holds columns [col0, col0 + vocab)
+    // of every row; instead of a score the row's (max, sum exp) pair and target logit go out
+    float2* pairs_out;         // [rows][pair_stride]
+    float* target_out;         // [rows]
+    int64_t pair_stride;
+    int64_t col0;
+    int64_t vocab;             // columns streamed per row
     int64_t row_stride;
     int32_t n_streams, max_new, n_part, logits_dtype, capacity;
 };
@@ -83,6 +91,7 @@ struct SelectParams {
     int32_t* keep_idx;
     int32_t* n_keep;
     int32_t* first_moved;
+    int32_t* ready;   // [n_streams] 1 once the stream's keep list, n_keep and first_moved are out
     int32_t* status;
     int32_t* epoch;
     unsigned long long* ticket;  // hand-out counter of the gather that follows: reset with the epoch
@@ -113,6 +122,7 @@ struct CompactParams {
     const int32_t* keep_idx;
     const int32_t* n_keep;
     const int32_t* first_moved;
+    int32_t* ready;        // [n_streams] raised by the preceding kernel once a stream's list is out
     int32_t* status;
     int32_t* epoch;        // bumped once per compaction by the kernel that precedes it
     unsigned long long* ticket;  // next work unit to hand out; zeroed by the same kernel
@@ -237,6 +247,14 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 // relaxed: a release store would first wait for every load the thread still has in flight.
 __device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void st_relaxed_u32(int32_t* p, uint32_t v) {
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_acquire_u32(const int32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
 
 // Order-preserving map from fp32 bit patterns to unsigned integers: a larger key is a

@@ -43,11 +43,13 @@ namespace {
 
 constexpr int kChunkRows = 32;  // rows per chunk = one per lane
 constexpr int kStoreSlack = 1;  // bulk stores that may still be reading shared memory
-constexpr int kMaxStages = 12;
+constexpr int kMaxStages = 8;
 constexpr int kIdxAhead = 4;     // chunks whose source indices are fetched ahead
 constexpr int kMaxWorkers = 4;   // worker warps per CTA
 constexpr int kPublishEvery = 4; // chunks between two updates of a segment's progress word
 constexpr int kNoBound = 0x7FFFFFFF;
+constexpr int kUnitsPerWorker = 28;  // work units per worker the split of the planes aims at
+constexpr int64_t kSmallJobBytes = 8 << 20;  // planes x longest keep list x row: the two-phase kernel's range
 
 // What the store of a chunk needs to know about the chunk ...
 struct StageInfo {
@@ -144,6 +146,24 @@ __device__ __forceinline__ bool store_chunk(uint64_t* full, const StageInfo* inf
     return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
 }
 
+// One warp waits (bounded) until the ready words of all n_streams streams are up.
+__device__ __forceinline__ bool wait_until_ready(const int32_t* ready, int n_streams, int lane) {
+    int ok = 1;
+    for (int s = lane; s < n_streams && ok; s += 32) {
+        uint32_t polls = 0;
+        while (ld_acquire_u32(&ready[s]) != 1u) {
+            if (++polls > kSpinLimit) {
+                ok = 0;
+                break;
+            }
+            if (polls > 64) __nanosleep(100);  // the word usually flips within a few microseconds
+        }
+    }
+    ok = __all_sync(0xFFFFFFFFu, ok);
+    __syncwarp();
+    return ok != 0;
+}
+
 __host__ __device__ inline size_t header_bytes(int n_workers) {
     const size_t h = (size_t)n_workers * kMaxStages * (8 + sizeof(StageInfo) + sizeof(UnitInfo));
     return (h + 127) & ~(size_t)127;
@@ -172,19 +192,31 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
         mbar_init_fence();
     }
     __syncwarp();
-    grid_dependency_wait();  // the keep lists, the epoch and the ticket counter of the preceding kernel
 
-    const uint32_t epoch = (uint32_t)*p.epoch;
+    // The kernel that precedes this one on the stream (selection, or the check of a caller's
+    // keep lists) raises ready[s] as soon as stream s's keep list and counts - and, with stream
+    // 0, the epoch and the ticket counter - are out, possibly long before it ends.  Under a
+    // programmatic dependent launch this grid polls those words instead of waiting for the whole
+    // preceding grid, so the gather starts while that kernel finishes its other work.  Every
+    // stream's word is awaited before anything that kernel wrote is read (lane i takes streams
+    // i, i + 32, ...), so those reads may go through L1.
+    bool alive = wait_until_ready(p.ready, (int)(p.planes_per_tensor / p.planes_per_stream), lane);
+
+    const uint32_t epoch = alive ? (uint32_t)*p.epoch : 0u;
     const int lead = stages - 1 - kStoreSlack;  // chunks whose loads run ahead of the stores
     const int64_t n_units = (int64_t)units_base * split;
     int64_t it = 0;      // chunks whose loads were issued
     int64_t stored = 0;  // chunks whose store was issued
     uint32_t unit_no = 0;
-    bool alive = true;
     SafeBound safe;
 
-    unsigned long long drawn = 0;  // lane 0: the number of the next unit
-    if (lane == 0) drawn = atomicAdd(p.ticket, 1ull);
+    // The first numbers are drawn once per CTA for all its workers (a quarter of the counter
+    // traffic while the whole grid starts at once), later ones by each worker for itself.
+    __shared__ unsigned long long first_ticket;
+    if (threadIdx.x == 0) first_ticket = alive ? atomicAdd(p.ticket, (unsigned long long)n_workers) : ~0ull;
+    __syncthreads();
+    unsigned long long drawn = first_ticket == ~0ull ? ~0ull : first_ticket + wid;  // lane 0's copy counts
+    alive = alive && drawn != ~0ull;
     while (alive) {
         const int64_t u = (int64_t)__shfl_sync(0xFFFFFFFFu, drawn, 0);
         if (u >= n_units) break;
@@ -301,7 +333,76 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
                 (void)mbar_wait_bounded(&full[c % stages], (uint32_t)((c / stages) & 1), kMbarSpinLimit);
         }
         bulk_wait_all();
+        // this grid must not be complete before the one it depends on is (what follows on the
+        // stream may rely on both); in practice that kernel ended long ago
+        grid_dependency_wait();
     }
+}
+
+// Small jobs (a few MB in all: short caches on few planes).  The ring above needs a long run
+// of chunks per worker to reach its speed and fills an SM's shared memory per CTA; here one CTA
+// takes one column slice of one plane and moves it in two phases - every moved row piece is
+// loaded into shared memory with 128-bit loads, the block synchronises, every piece is stored -
+// so no store can overtake a load, in place or not, and slices (whole 32-byte sectors of a
+// row) never touch each other's bytes.  Chosen by the host when all of a slice fits in shared
+// memory and the job is too small to fill the persistent grid.
+constexpr int kSmallThreads = 256;
+
+__global__ void __launch_bounds__(kSmallThreads)
+compact_small_kernel(const CompactParams p, const int col_splits) {
+    extern __shared__ uint4 staged[];
+    __shared__ int sh_ok;
+    const int r = (int)(blockIdx.x / col_splits), c = (int)(blockIdx.x - (unsigned)r * col_splits);
+    const int tensor = (int)(r / p.planes_per_tensor);
+    const int64_t plane = r - (int64_t)tensor * p.planes_per_tensor;
+    const int s = (int)(plane / p.planes_per_stream);
+    if (threadIdx.x < 32) {  // the keep lists are out (see compact_kernel)
+        const bool ok = wait_until_ready(p.ready, (int)(p.planes_per_tensor / p.planes_per_stream), threadIdx.x);
+        if (threadIdx.x == 0) {
+            if (!ok) atomicOr(p.status, SIRLLM_STATUS_TIMEOUT);
+            sh_ok = ok;
+        }
+    }
+    __syncthreads();
+    if (sh_ok) {
+        const int n = min(max(p.n_keep[s], 0), p.keep_stride);
+        int f = p.first_moved[s];
+        if (!p.in_place && f >= 0) f = 0;
+        if (f >= 0 && f < n) {
+            const int row_vecs = p.row_bytes / 16, slice_vecs = row_vecs / col_splits;
+            const uint4* src = reinterpret_cast<const uint4*>(
+                (tensor ? p.src[1] : p.src[0]) + (size_t)plane * p.capacity * p.row_bytes) + c * slice_vecs;
+            uint4* dst = reinterpret_cast<uint4*>(
+                (tensor ? p.dst[1] : p.dst[0]) + (size_t)plane * p.capacity * p.row_bytes) + c * slice_vecs;
+            const int32_t* keep = p.keep_idx + (size_t)s * p.keep_stride;
+            const int total = (n - f) * slice_vecs;
+            constexpr int kBatch = 4;  // independent loads in flight per thread
+            for (int base = 0; base < total; base += kBatch * kSmallThreads) {
+                int kj[kBatch];
+#pragma unroll
+                for (int q = 0; q < kBatch; ++q) {
+                    const int i = base + q * kSmallThreads + threadIdx.x;
+                    kj[q] = i < total ? keep[f + i / slice_vecs] : 0;
+                }
+                uint4 x[kBatch];
+#pragma unroll
+                for (int q = 0; q < kBatch; ++q) {
+                    const int i = base + q * kSmallThreads + threadIdx.x;
+                    if (i < total) x[q] = src[(size_t)kj[q] * row_vecs + i % slice_vecs];
+                }
+#pragma unroll
+                for (int q = 0; q < kBatch; ++q) {
+                    const int i = base + q * kSmallThreads + threadIdx.x;
+                    if (i < total) staged[i] = x[q];
+                }
+            }
+            __syncthreads();  // every source row of the slice has been read
+            for (int i = threadIdx.x; i < total; i += kSmallThreads)
+                dst[(size_t)(f + i / slice_vecs) * row_vecs + i % slice_vecs] = staged[i];
+        }
+    }
+    // not complete before the grid this one depends on is (see compact_kernel)
+    if (threadIdx.x == 0) grid_dependency_wait();
 }
 
 // Checks caller-supplied keep lists and finds, per stream, the first slot whose row moves.
@@ -333,6 +434,8 @@ __global__ void compact_plan_kernel(const CompactParams p, int32_t* __restrict__
         } else {
             first_moved[s] = sh_first;
         }
+        __threadfence();
+        st_relaxed_u32(&p.ready[s], 1u);  // the gather polls this word
     }
 }
 
@@ -392,10 +495,41 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     if (e != cudaSuccess) return e;
 
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+
+    // a job too small to fill the persistent grid goes to the two-phase kernel: one CTA per
+    // plane and column slice (slices of at least 32 bytes, as many as it takes to occupy the
+    // SMs), provided a slice of the longest keep list fits in shared memory
+    const int row_vecs = p.row_bytes / 16;
+    if ((int64_t)units_base * p.keep_stride * p.row_bytes <= kSmallJobBytes) {
+        int col_splits = 1;
+        while (col_splits * 2 <= row_vecs / 2 && row_vecs % (col_splits * 2) == 0 &&
+               (int64_t)units_base * col_splits < 2 * n_sm)
+            col_splits *= 2;
+        const size_t small_smem = (size_t)p.keep_stride * (p.row_bytes / col_splits);
+        if (small_smem <= (size_t)smem_max - 1024) {
+            e = cudaFuncSetAttribute(compact_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)small_smem);
+            if (e != cudaSuccess) return e;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)(units_base * col_splits));
+            cfg.blockDim = dim3(kSmallThreads);
+            cfg.dynamicSmemBytes = small_smem;
+            cfg.stream = st;
+            cfg.attrs = attr;
+            cfg.numAttrs = overlap ? 1 : 0;
+            return cudaLaunchKernelEx(&cfg, compact_small_kernel, q, col_splits);
+        }
+    }
+
     // ring geometry: kMaxWorkers workers per CTA with 6 to 8 stages each; fewer workers, then
     // fewer stages (at least 4), when the rows are too wide for that
     const size_t stage_bytes = (size_t)kChunkRows * p.row_bytes;
-    const size_t budget = (size_t)smem_max - 2048;
+    // what is left for the rings beside the records in front of them and the kernel's few
+    // bytes of static shared memory
+    const size_t budget = (size_t)smem_max - header_bytes(kMaxWorkers) - 256;
     int workers = kMaxWorkers, stages = 6;
     while (workers > 1 && (size_t)workers * stages * stage_bytes > budget) --workers;
     while (stages > 4 && (size_t)workers * stages * stage_bytes > budget) --stages;
@@ -412,21 +546,18 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     if (e != cudaSuccess) return e;
     if (per_sm < 1) return cudaErrorLaunchOutOfResources;
     const int64_t resident = (int64_t)n_sm * per_sm;
-    // cut planes into segments so that the units spread evenly over the workers: fewest idle
-    // worker-rounds, then fewest segments
+    // Cut planes into segments so that every worker draws a few dozen units: the ticket
+    // hand-out then evens out SMs of different speed down to a small tail, while a unit stays
+    // long enough (at least four chunks at the longest keep list) to amortise its set-up.
+    // About 28 units per worker measured best on every shape tried (14 and 55 were worse).
     const int64_t slots = resident * workers;
     int split = 1;
-    if (units_base < 8 * slots && units_base <= kChainPlanesMax) {
-        double best = -1.0;
-        for (int h = 1; h <= kMaxSplit; ++h) {
-            const int64_t units = (int64_t)units_base * h;
-            const int64_t rounds = (units + slots - 1) / slots;
-            const double eff = (double)units / (double)(rounds * slots);
-            if (eff > best + 0.02) {
-                best = eff;
-                split = h;
-            }
-        }
+    if (units_base <= kChainPlanesMax) {
+        const int64_t chunks_max = (p.keep_stride + kChunkRows - 1) / kChunkRows;
+        int64_t want_split = (kUnitsPerWorker * slots + units_base / 2) / units_base;
+        if (want_split > chunks_max / 4) want_split = chunks_max / 4;
+        if (want_split > kMaxSplit) want_split = kMaxSplit;
+        if (want_split > 1) split = (int)want_split;
     }
     const int64_t n_units = (int64_t)units_base * split;
     const int64_t want = (n_units + workers - 1) / workers;
@@ -436,9 +567,6 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     cfg.blockDim = dim3((unsigned)workers * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, compact_kernel, q, stages, units_base, split);

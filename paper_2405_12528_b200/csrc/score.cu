@@ -64,6 +64,8 @@ score_kernel(const ScoreParams p) {
     constexpr int EPV = 16 / ES;
     __shared__ float2 warp_pair[kWarps];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    // the selection kernel may become resident while this grid drains (it waits for this grid's
+    // scores itself); this grid starts only after everything before it on the stream is complete
     grid_launch_dependents();
     // one CTA = kWarps consecutive segments of one logits row
     const int64_t row = blockIdx.x / p.n_part;
@@ -200,7 +202,21 @@ score_kernel(const ScoreParams p) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
     }
-    if (lane == 0) {
+    if (lane == 0 && p.pairs_out != nullptr) {
+        // vocabulary-parallel: hand over this column range's share of the row's softmax sum as
+        // (m, s) with sum_v exp z_v = s * exp(m), m within rounding of the range's maximum
+        // (natural units), and the target logit if the token's column lies in the range
+        float2 pr = make_float2(0.f, 0.f);  // an empty or fully masked range contributes nothing
+        if (acc > 0.0) {
+            pr.x = (float)((double)Mx * kLn2);
+            pr.y = (float)(acc * exp2((double)Mx - (double)pr.x * 1.4426950408889634));
+        }
+        p.pairs_out[row * p.pair_stride] = pr;
+        const int64_t col = (int64_t)id - p.col0;
+        p.target_out[row] = (id >= 0 && col >= 0 && col < V)
+                                ? load_logit(rowp, kBf16 ? SIRLLM_BF16 : SIRLLM_F32, col)
+                                : 0.f;
+    } else if (lane == 0) {
         // e = ln(sum_v exp z_v) - z_id >= 0; id -1 = no prediction, other bad ids are flagged
         float e = 0.f;
         if (id >= 0 && (int64_t)id < V) {
@@ -270,6 +286,9 @@ cudaError_t launch_score_pairs(const PairScoreParams& p, cudaStream_t st) {
     return cudaGetLastError();
 }
 
+// Launched plainly: the grid starts once everything before it on the stream is complete.  (A
+// programmatic launch that let it become resident during the preceding gather was measured:
+// the parked CTAs slowed the gather by 2-3 %, and short rounds by more.)
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
     const int64_t ctas = (int64_t)p.n_streams * p.max_new * p.n_part;
     if (ctas == 0) return cudaSuccess;
@@ -374,6 +393,10 @@ extern "C" int sirllm_score_static(const sirllm_config* cfg, const void* logits,
     sp.out_entropy = out_entropy;
     sp.scores = nullptr;
     sp.live_len = nullptr;
+    sp.pairs_out = nullptr;
+    sp.target_out = nullptr;
+    sp.pair_stride = 0;
+    sp.col0 = 0;
     sp.vocab = cfg->vocab;
     sp.row_stride = cfg->logits_row_stride;
     sp.n_streams = cfg->n_streams;

@@ -65,6 +65,20 @@ __device__ __forceinline__ int block_inclusive_scan(int v, uint32_t* warp_sum) {
     return (int)block_inclusive_scan_u32((uint32_t)v, warp_sum);
 }
 
+// The keep list of stream s is complete: make it (and the counts) visible to the whole GPU and
+// raise the stream's ready word, which the KV gather that follows polls instead of waiting for
+// this whole grid to finish - compaction of K and V then overlaps the rest of this kernel
+// (score and tag compaction).  Called by every thread of the block, on every path.
+__device__ __forceinline__ void publish_keep_list(const SelectParams& p, int s, int n_keep, int first_moved) {
+    __syncthreads();  // every thread's part of the keep list precedes ...
+    if (threadIdx.x == 0) {
+        p.n_keep[s] = n_keep;
+        p.first_moved[s] = first_moved;
+        __threadfence();  // ... this fence (cumulative), and so the word raised after it
+        st_relaxed_u32(&p.ready[s], 1u);
+    }
+}
+
 // kStage: the keep list is assembled in shared memory and written out coalesced (the host
 // chooses this whenever capacity + threshold words fit); otherwise it goes straight to global
 // memory from the owning threads.
@@ -81,6 +95,12 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     const int cap = p.capacity;
     float* scores = p.scores + (size_t)s * cap;
     int32_t* keep = p.keep_idx + (size_t)s * p.threshold;
+    // the gather polls ready[s]: take it down before any dependent grid can start
+    if (tid == 0) {
+        st_relaxed_u32(&p.ready[s], 0u);
+        __threadfence();
+    }
+    __syncthreads();
     grid_launch_dependents();
     // In the fused round this grid may become resident while the scorer is still draining
     // (programmatic dependent launch).  Everything up to grid_dependency_wait() uses only
@@ -102,10 +122,9 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
                 *p.ticket = 0ull;
             }
             atomicOr(p.status, SIRLLM_STATUS_OVERFLOW);
-            const int n = max(0, min(l0, min(cap, p.threshold)));
-            p.n_keep[s] = n;
-            p.first_moved[s] = n;
         }
+        const int n = max(0, min(l0, min(cap, p.threshold)));
+        publish_keep_list(p, s, n, n);  // nothing moves
         return;
     }
     const int l = l0 + T;
@@ -151,11 +170,8 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     decay_range(l0, l);      // this round's scores
     if (!evict) {  // ---- nothing to evict: identity keep list --------------------------
         for (int i = tid; i < l; i += kSelectThreads) keep[i] = i;
-        if (tid == 0) {
-            p.n_keep[s] = l;
-            p.first_moved[s] = l;
-            if (p.compact_scores) p.live_len[s] = l;
-        }
+        publish_keep_list(p, s, l, l);
+        if (tid == 0 && p.compact_scores) p.live_len[s] = l;
         return;
     }
 
@@ -320,12 +336,12 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     if (lane == 0 && my_first_evicted < l) atomicMin(&sh.first_evicted, my_first_evicted);
     __syncthreads();
     const int first = sh.first_evicted;
-    if (kStage) {  // coalesced copy-out of the list and of the scores it selects
-        for (int j = tid; j < p.budget; j += kSelectThreads) {
-            const int src = skeep[j];
-            keep[j] = src;
-            if (p.compact_scores) scores[j] = __uint_as_float(vals[src]);
-        }
+    if (kStage) {  // coalesced copy-out of the list ...
+        for (int j = tid; j < p.budget; j += kSelectThreads) keep[j] = skeep[j];
+    }
+    publish_keep_list(p, s, p.budget, first);  // the KV gather may start
+    if (kStage && p.compact_scores) {  // ... and of the scores it selects
+        for (int j = tid; j < p.budget; j += kSelectThreads) scores[j] = __uint_as_float(vals[skeep[j]]);
     }
 
     // ---- S5: the 8-byte tags follow, in place, front to back.  A batch of kTagBatch tags
@@ -350,11 +366,7 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
             __syncthreads();
         }
     }
-    if (tid == 0) {  // ---- S7
-        p.n_keep[s] = p.budget;
-        p.first_moved[s] = first;
-        if (p.compact_scores) p.live_len[s] = p.budget;
-    }
+    if (tid == 0 && p.compact_scores) p.live_len[s] = p.budget;  // ---- S7
 }
 
 }  // namespace

@@ -443,6 +443,108 @@ def test_step_pairs_round_matches_oracle_and_the_logits_round():
         b.check_kv_by_content()
 
 
+# ------------------------------------------------------------------------------- sharded forms
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_score_partial_over_uneven_column_ranges_matches_oracle(dtype):
+    # a vocabulary-parallel LM head: every "rank" (here: one call each, on one device) reduces
+    # its column range to a pair and a target logit per row; the pairs of all ranges then give
+    # the scores.  Ranges are uneven, start off the 16-byte grid, one is empty, one is a few
+    # columns wide and one needs several CTAs per row.
+    S, M, V = 2, 30, 70001
+    ranges = [(0, 5), (5, 40001), (40001, 40001), (40001, V)]
+    cfg = _score_cfg(M, V, dtype, n_streams=S)
+    ws = B.new_workspace(cfg)
+    g = torch.Generator().manual_seed(3)
+    logits = (torch.randn(S * M, V, generator=g) * 2.5).to(dtype)
+    logits[4, 10:30000] = -float("inf")                   # masked stretch inside one range
+    ids = torch.randint(0, V, (S * M,), generator=g, dtype=torch.int32)
+    ids[1], ids[2], ids[5], ids[6] = -1, 3, 40000, 40001  # no prediction; range edges
+    n_new = torch.tensor([M, 11], dtype=torch.int32)
+    d_logits, d_ids, d_n = logits.to(DEV), ids.to(DEV), n_new.to(DEV)
+    pairs = torch.full((S * M, len(ranges), 2), -9.0, device=DEV)
+    targets = torch.full((len(ranges), S * M), -9.0, device=DEV)
+    for r, (v0, v1) in enumerate(ranges):
+        B.sirllm_score_partial(cfg, d_logits[:, v0:v1], v0, d_ids, d_n, pairs, targets[r], ws, pair_column=r)
+    live = torch.zeros(S * M, dtype=torch.bool)
+    live[:M] = True
+    live[M:M + 11] = True
+    assert (pairs.cpu()[~live] == -9.0).all() and (targets.cpu()[:, ~live] == -9.0).all()
+    for r, (v0, v1) in enumerate(ranges):                 # each range against the oracle's pair
+        want_p, want_t = oracle.range_pairs(logits, ids, v0, v1)
+        got_p = pairs[:, r].cpu()
+        assert torch.equal(targets[r].cpu()[live], want_t[live])
+        empty = want_p[:, 1] == 0
+        assert (got_p[empty & live] == 0).all()
+        ok = live & ~empty
+        if not ok.any():
+            continue
+        lse_got = got_p[ok, 0].double() + got_p[ok, 1].double().log()     # log of the range's sum
+        lse_want = want_p[ok, 0].double() + want_p[ok, 1].double().log()
+        assert float((lse_got - lse_want).abs().max()) < 2e-6
+        assert float((got_p[ok, 0] - want_p[ok, 0]).abs().max()) < 1e-5   # m ~ the range's maximum
+    target = targets.clone()
+    target[:, ~live.to(DEV)] = 0
+    target = target.sum(dim=0)
+    out = torch.full((S * M,), -2.0, device=DEV)
+    B.sirllm_score_pairs(cfg, pairs, target, d_ids, d_n, out, ws)
+    assert B.sirllm_status(ws) == 0
+    want = oracle.score(logits, ids)
+    assert_entropy_close(out.cpu()[live], want[live])
+    ref = torch.zeros(S * M, device=DEV)                  # and against the single-GPU kernel
+    B.sirllm_score(cfg, d_logits, d_ids, d_n, ref, ws)
+    assert_entropy_close(out.cpu()[live], ref.cpu()[live])
+
+
+@pytest.mark.parametrize("by", ["layers", "heads"])
+def test_plane_sharded_rounds_equal_the_full_configuration(by):
+    # tensor- / pipeline-parallel layouts: every rank holds a replica of the scores and the K/V
+    # planes of some layers or heads.  Two such ranks (run one after the other on one device),
+    # each with its own workspace and its own half of the planes, must produce the keep lists,
+    # scores and tags of the unsharded run and, between them, its K/V - all of it the oracle's.
+    from paper_2405_12528_b200 import sharding
+    w = wl.WORKLOADS["mistral_7b_gqa"].scaled(n_streams=2, n_layers=4, n_kv_heads=2, capacity=768,
+                                              budget=512, n_recent=64, new_tokens=150, vocab=4001)
+    full = DeviceState(w)
+    twins = oracle_twin(w, full.decay.cpu(), with_kv=False)
+    world = 2
+    ranks = []
+    for r in range(world):
+        layers, heads = sharding.plane_shard(w.n_layers, w.n_kv_heads, world, r, by)
+        st = DeviceState(w.scaled(n_layers=len(layers), n_kv_heads=len(heads)))
+        planes = torch.tensor([l * w.n_kv_heads + h for l in layers for h in heads], device=DEV)
+        ranks.append((st, planes))
+    for rnd in range(8):
+        n_new = full.fill_round(rnd, wl.ragged_lengths(5, w.n_streams, rnd, w.new_tokens).tolist())
+        for st, planes in ranks:                          # the same round on every rank
+            st.logits.copy_(full.logits)
+            st.token_ids.copy_(full.token_ids)
+            st.n_new.copy_(full.n_new)
+            for s in range(w.n_streams):
+                l, T = st.host_len[s], n_new[s]
+                st.serial[s, l:l + T] = full.serial[s, l:l + T]
+                st.k[s, :, l:l + T] = full.k[s, planes, l:l + T]
+                st.v[s, :, l:l + T] = full.v[s, planes, l:l + T]
+        full.step()
+        for st, _ in ranks:
+            st.step()
+            assert B.sirllm_status(st.ws) == 0 and st.host_len == full.host_len
+        e = full.new_entropy.cpu()
+        M = full.cfg.max_new
+        for s, tw in enumerate(twins):
+            n = full.host_len[s]
+            for st, planes in ranks:
+                assert torch.equal(st.keep_idx[s, :n], full.keep_idx[s, :n])
+                assert torch.equal(st.scores[s, :n].view(torch.int32), full.scores[s, :n].view(torch.int32))
+                assert torch.equal(st.serial[s, :n], full.serial[s, :n])
+                assert torch.equal(st.k[s, :, :n], full.k[s, planes, :n])
+                assert torch.equal(st.v[s, :, :n], full.v[s, planes, :n])
+            keep = tw.step(e[s * M:s * M + n_new[s]])     # the oracle ranks the same scores
+            assert tw.live_len == n and torch.equal(full.keep_idx[s, :n].cpu(), keep)
+            assert torch.equal(full.scores[s, :n].cpu().view(torch.int32), tw.E[:n].view(torch.int32))
+        full.check_kv_by_content()                        # K/V rows follow their tokens
+
+
 # ------------------------------------------------------------------------------- comparison policies
 
 @pytest.mark.parametrize("policy", [B.POLICY_STREAM, B.POLICY_RANDOM, B.POLICY_INTERVAL])

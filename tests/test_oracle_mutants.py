@@ -29,6 +29,15 @@ MUTANTS = {
         ("return (m - logit_at(row, dtype, id)) + log(s);", "return (m - m) + log(s);"),
     "pairs: tile maxima ignored":
         ("S += (double)pairs[2 * i + 1] * exp((double)pairs[2 * i] - M);", "S += (double)pairs[2 * i + 1];"),
+    "range pair: every rank claims the target logit":
+        ("(id >= 0 && (int64_t)id >= v0 && (int64_t)id < v1) ? (float)logit_at(row, dtype, id) : 0.0f;",
+         "(id >= 0) ? (float)logit_at(row, dtype, id) : 0.0f;"),
+    "range pair: sum not taken relative to the range's maximum":
+        ("        for (int64_t v = v0; v < v1; ++v)\n            s += exp(logit_at(row, dtype, v) - m);",
+         "        for (int64_t v = v0; v < v1; ++v)\n            s += exp(logit_at(row, dtype, v));"),
+    "range pair: maximum of the whole row":
+        ("    for (int64_t v = v0; v < v1; ++v) {\n        double z = logit_at(row, dtype, v);",
+         "    for (int64_t v = 0; v < v1; ++v) {\n        double z = logit_at(row, dtype, v);"),
     "decay: applied to the old scores only":
         ("    l += T;\n    oracle_decay(E, l, eta);", "    oracle_decay(E, l, eta);\n    l += T;"),
     "decay: applied twice per round":

@@ -66,3 +66,51 @@ def test_invariances():
     rs[:, 5, 0] += math.log(2.0)
     rs[:, 5, 1] /= 2.0
     assert torch.allclose(oracle.score_pairs(rs.float(), target, ids, 10).double(), base, atol=1e-6)
+
+
+# ---- one rank's column range (vocabulary-parallel LM head) ---------------------------------
+
+@pytest.mark.parametrize("cuts", [[0, 3001], [0, 1, 3001], [0, 1500, 3001], [0, 7, 7, 2999, 3000, 3001],
+                                  [0, 1024, 2048, 3001], [0, 0, 3001, 3001]])
+def test_uneven_column_ranges_give_the_same_entropy_as_the_whole_row(cuts):
+    # any cutting of the vocabulary into contiguous ranges - uneven, single-column, empty - must
+    # reproduce the whole-row definition once the ranges' pairs are combined
+    g = torch.Generator().manual_seed(len(cuts))
+    for dtype in (torch.float32, torch.bfloat16):
+        logits = (torch.randn(7, 3001, generator=g) * 3).to(dtype)
+        logits[2, 100:900] = -float("inf")                      # a stretch of masked columns
+        ids = torch.randint(0, 3001, (7,), generator=g, dtype=torch.int32)
+        ids[2] = 950
+        ids[3] = -1
+        parts = [oracle.range_pairs(logits, ids, a, b) for a, b in zip(cuts[:-1], cuts[1:])]
+        pairs = torch.stack([p for p, _ in parts], dim=1)       # [T, ranks, 2]
+        target = torch.stack([t for _, t in parts]).sum(dim=0)  # only the owning range is non-zero
+        assert torch.equal(target[ids >= 0], logits.float()[torch.arange(7), ids.long().clamp(min=0)][ids >= 0])
+        got = oracle.score_pairs(pairs, target, ids, 3001)
+        want = oracle.score(logits, ids)
+        np.testing.assert_allclose(got.numpy(), want.numpy(), rtol=0, atol=2e-6)
+        assert float(got[3]) == 0.0
+
+
+def test_range_pair_closed_forms():
+    # n equal logits c in the range: (c, n); a fully masked or empty range: (0, 0)
+    row = torch.full((1, 64), 1.25)
+    row[0, 40:] = -float("inf")
+    ids = torch.tensor([5], dtype=torch.int32)
+    p, t = oracle.range_pairs(row, ids, 0, 32)
+    assert p.tolist() == [[1.25, 32.0]] and t.tolist() == [1.25]
+    p, t = oracle.range_pairs(row, ids, 32, 64)                 # 8 live columns, 24 masked
+    assert p.tolist() == [[1.25, 8.0]] and t.tolist() == [0.0]
+    p, t = oracle.range_pairs(row, ids, 40, 64)
+    assert p.tolist() == [[0.0, 0.0]]
+    p, t = oracle.range_pairs(row, ids, 10, 10)
+    assert p.tolist() == [[0.0, 0.0]] and t.tolist() == [0.0]
+    # the maximum is the range's own, whatever the rest of the row holds
+    row = torch.cat([torch.full((1, 32), 5.0), torch.full((1, 32), 1.25)], dim=1)
+    p, _ = oracle.range_pairs(row, ids, 32, 64)
+    assert p.tolist() == [[1.25, 32.0]]
+    # two columns (0, ln 3): max ln 3, sum 1 + 1/3
+    row = torch.tensor([[0.0, math.log(3.0)]])
+    p, _ = oracle.range_pairs(row, torch.tensor([0], dtype=torch.int32), 0, 2)
+    assert float(p[0, 0]) == pytest.approx(math.log(3.0), abs=1e-7)
+    assert float(p[0, 1]) == pytest.approx(4.0 / 3.0, abs=1e-7)

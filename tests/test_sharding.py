@@ -77,3 +77,62 @@ def test_two_ranks_shard_streams_and_reduce_only_bookkeeping():
         assert len(set(single)) > 1                     # and the streams really differ
         assert slowest == 3.0                           # max over ranks
         assert tokens == 4 * 96                         # whole-job count
+
+
+# ---- vocabulary-parallel scoring: the exchange, with the oracle standing in for the GPUs ----
+
+def _vocab_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        w = wl.WORKLOADS["tiny"].scaled(new_tokens=40, vocab=1001)
+        logits = wl.make_logits(w, 0, 0, 0)
+        ids = wl.make_token_ids(w, 0, 0, 0)
+        ids[3] = -1
+        v0, v1 = sharding.vocab_ranges(w.vocab, world)[rank]
+        # this rank only ever looks at its own columns
+        pairs_local, target_local = oracle.range_pairs(logits[:, v0:v1].contiguous(), ids - v0 * (ids >= 0),
+                                                       0, v1 - v0)
+        pairs, target = sharding.exchange_vocab_partials(pairs_local, target_local)
+        e = oracle.score_pairs(pairs, target, ids, w.vocab)
+        out.put((rank, tuple(pairs.shape), e.tolist()))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_vocab_ranges_cover_the_vocabulary():
+    for vocab, world in ((32000, 8), (128256, 3), (5, 8), (1001, 2)):
+        r = sharding.vocab_ranges(vocab, world)
+        assert r[0][0] == 0 and r[-1][1] == vocab and len(r) == world
+        assert all(a[1] == b[0] for a, b in zip(r[:-1], r[1:]))
+        assert max(b - a for a, b in r) - min(b - a for a, b in r) <= 1
+
+
+def test_two_ranks_score_a_vocabulary_split_across_them():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_vocab_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    w = wl.WORKLOADS["tiny"].scaled(new_tokens=40, vocab=1001)
+    ids = wl.make_token_ids(w, 0, 0, 0)
+    ids[3] = -1
+    want = oracle.score(wl.make_logits(w, 0, 0, 0), ids)
+    for rank, shape, e in results:
+        assert shape == (40, 2, 2)
+        assert e == results[0][2]                         # every rank ends with the same scores
+        assert torch.allclose(torch.tensor(e), want, rtol=0, atol=2e-6)
+        assert e[3] == 0.0
+
+
+def test_plane_shards_partition_the_planes():
+    for by, (L, H) in (("layers", (32, 8)), ("heads", (32, 8)), ("layers", (5, 3))):
+        for world in (1, 2, 4):
+            owned = [sharding.plane_shard(L, H, world, r, by) for r in range(world)]
+            planes = sorted((l, h) for ls, hs in owned for l in ls for h in hs)
+            assert planes == [(l, h) for l in range(L) for h in range(H)]
