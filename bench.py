@@ -157,6 +157,10 @@ class Pass:
             self.pool.append((lg, ids))
         self.next_serial = 0
         self.round = 0
+        # the fused round on either logits tensor, arguments checked and marshalled once
+        self.fused = [B.prepared(B.sirllm_step, self.cfg, lg, ids, self.n_new, self.scores, self.serial,
+                                 self.live_len, self.decay, self.k, self.v, self.keep_idx, self.n_keep,
+                                 self.new_entropy, self.ws) for lg, ids in self.pool]
 
     def append_rows(self):
         """Stand-in for the model: writes the round's new K/V rows and tags behind the live rows."""
@@ -172,14 +176,15 @@ class Pass:
         self.next_serial += T
 
     def step(self, events=None):
-        lg, ids = self.pool[self.round & 1]
+        which = self.round & 1
         self.round += 1
-        args = (self.cfg, lg, ids, self.n_new, self.scores, self.serial, self.live_len, self.decay,
-                self.k, self.v, self.keep_idx, self.n_keep, self.new_entropy, self.ws)
         if events is None:
-            self.B.sirllm_step(*args)
+            self.fused[which]()
         else:
-            self.B.sirllm_step_phases(*args, events)
+            lg, ids = self.pool[which]
+            self.B.sirllm_step_phases(self.cfg, lg, ids, self.n_new, self.scores, self.serial,
+                                      self.live_len, self.decay, self.k, self.v, self.keep_idx,
+                                      self.n_keep, self.new_entropy, self.ws, events)
 
     def prime(self):
         """Real rounds from an empty cache until the first eviction has happened."""

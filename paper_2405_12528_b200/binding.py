@@ -9,6 +9,7 @@ from __future__ import annotations
 
 import ctypes
 import os
+import threading
 from typing import Optional
 
 import torch
@@ -183,14 +184,58 @@ def _dev(t, dtype=None, name="tensor", numel: int = 0) -> _Arg:
     return _Arg(t, dtype, name, numel)
 
 
+class Prepared:
+    """A call whose arguments were checked and marshalled once (see :func:`prepared`): calling
+    it again costs one ctypes call.  It keeps its tensors alive and reads the current CUDA
+    stream at every call; it must be called with the device it was prepared on current."""
+
+    def __init__(self, fn, cfg, args):
+        self._fn, self._cfg = fn, Config.from_buffer_copy(cfg)
+        self._keep = [a.t for a in args if isinstance(a, _Arg)]
+        self._raw = [a.ptr() if isinstance(a, _Arg) else a for a in args]
+        self._stream_at = [i for i, a in enumerate(args) if isinstance(a, _CurrentStream)]
+        self._cfg_ref = ctypes.byref(self._cfg)
+
+    def __call__(self) -> None:
+        raw = self._raw
+        for i in self._stream_at:
+            raw[i] = torch.cuda.current_stream().cuda_stream
+        rc = self._fn(self._cfg_ref, *raw)
+        if rc != OK:
+            _check(rc)
+
+
+_preparing = threading.local()
+
+
+def prepared(func, *args, **kwargs) -> Prepared:
+    """``prepared(sirllm_step, cfg, logits, ...)`` checks and marshals the arguments of one of
+    this module's calls once and returns a :class:`Prepared` that issues exactly that call
+    (same tensors, whatever they hold by then) each time it is invoked - for loops that repeat
+    a call thousands of times a second, where the per-argument checks would dominate."""
+    _preparing.out = None
+    _preparing.on = True
+    try:
+        func(*args, **kwargs)
+    finally:
+        _preparing.on = False
+    if _preparing.out is None:
+        raise SirllmError(ERR_BAD_CONFIG, f"{getattr(func, '__name__', func)} cannot be prepared")
+    return _preparing.out
+
+
 def _call(fn, cfg, *args) -> None:
-    """Checks every tensor argument (shapes of all first, then residence), then calls ``fn``."""
+    """Checks every tensor argument (shapes of all first, then residence), then calls ``fn``
+    (or, under :func:`prepared`, hands back the marshalled call instead of making it)."""
     for a in args:
         if isinstance(a, _Arg):
             a.check_shape()
     for a in args:
         if isinstance(a, _Arg):
             a.check_residence()
+    if getattr(_preparing, "on", False):
+        _preparing.out = Prepared(fn, cfg, args)
+        return
     raw = [a.ptr() if isinstance(a, _Arg) else _stream_handle() if isinstance(a, _CurrentStream) else a
            for a in args]
     _check(fn(ctypes.byref(cfg), *raw))

@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in sirllm.h: argument checks, workspace layout and
 // the launch sequences.  No device memory is allocated here.
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -13,6 +14,43 @@ static thread_local char g_cuda_msg[256] = "";
 int cuda_fail(cudaError_t e, const char* where) {
     snprintf(g_cuda_msg, sizeof g_cuda_msg, "%s: %s", where, cudaGetErrorString(e));
     return SIRLLM_ERR_CUDA;
+}
+
+cudaError_t device_props(DeviceProps* out) {
+    static DeviceProps cache[kMaxDevices];
+    static std::atomic<int> known[kMaxDevices];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < kMaxDevices && known[dev].load(std::memory_order_acquire)) {
+        *out = cache[dev];
+        return cudaSuccess;
+    }
+    DeviceProps dp;
+    dp.device = dev;
+    e = cudaDeviceGetAttribute(&dp.n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&dp.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < kMaxDevices) {  // several threads may fill the slot: they write the same values
+        cache[dev] = dp;
+        known[dev].store(1, std::memory_order_release);
+    }
+    *out = dp;
+    return cudaSuccess;
+}
+
+cudaError_t allow_max_dynamic_smem(const void* kernel, const DeviceProps& dp, unsigned char* done) {
+    const bool cached = dp.device >= 0 && dp.device < kMaxDevices;
+    if (cached && __atomic_load_n(&done[dp.device], __ATOMIC_ACQUIRE)) return cudaSuccess;
+    cudaFuncAttributes fa;
+    cudaError_t e = cudaFuncGetAttributes(&fa, kernel);
+    if (e != cudaSuccess) return e;
+    // static and dynamic shared memory together may reach the opt-in limit
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             dp.smem_optin - (int)fa.sharedSizeBytes);
+    if (e == cudaSuccess && cached) __atomic_store_n(&done[dp.device], (unsigned char)1, __ATOMIC_RELEASE);
+    return e;
 }
 
 int validate_config(const sirllm_config* c) {

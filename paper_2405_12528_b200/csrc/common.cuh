@@ -43,6 +43,19 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int logits_elem_bytes(int dtype) { return dtype == SIRLLM_F32 ? 4 : 2; }
 
 int validate_config(const sirllm_config* cfg);
+
+// Properties of the current device that the launch code needs at every call, looked up once per
+// device and process (they never change): SM count and the opt-in shared-memory limit.
+struct DeviceProps {
+    int device;
+    int n_sm;
+    int smem_optin;
+};
+cudaError_t device_props(DeviceProps* out);
+// Raises a kernel's dynamic shared-memory limit to the device's opt-in maximum, once per device.
+// `done` is the kernel's own flag array (kMaxDevices entries, zero-initialised).
+constexpr int kMaxDevices = 64;
+cudaError_t allow_max_dynamic_smem(const void* kernel, const DeviceProps& dp, unsigned char* done);
 // Records the message sirllm_last_cuda_error() returns and yields SIRLLM_ERR_CUDA.
 int cuda_fail(cudaError_t e, const char* where);
 WorkspaceLayout workspace_layout(const sirllm_config& cfg);

@@ -35,6 +35,8 @@
 // smaller number than its own, and every smaller number was drawn by a worker that is
 // running (it drew the number itself), so by induction the waits end whatever number of CTAs
 // the device keeps resident at once.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace sirllm {
@@ -146,6 +148,46 @@ __device__ __forceinline__ bool store_chunk(uint64_t* full, const StageInfo* inf
     return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
 }
 
+// One work unit (a segment of the moved rows of one plane), resolved from its number.
+struct Unit {
+    const char* src;
+    char* dst;
+    const int32_t* keep;
+    unsigned long long* prog;  // progress words of the plane (chained units)
+    int j_begin, j_end;        // destination rows of the segment
+    int h, n_seg;              // segment index, segments of the plane
+    int f, n, seg_rows;        // first moved row, rows kept, rows per full segment
+    bool chained;              // in place and the plane has several segments
+    bool valid;                // false: nothing to move for this number
+};
+
+__device__ __forceinline__ Unit resolve_unit(const CompactParams& p, int64_t u, int units_base, int split) {
+    Unit un;
+    un.h = (int)(u / units_base);  // segment of the plane's moved rows
+    const int r = (int)(u - (int64_t)un.h * units_base);
+    const int tensor = (int)(r / p.planes_per_tensor);
+    const int64_t plane = r - (int64_t)tensor * p.planes_per_tensor;
+    const int s = (int)(plane / p.planes_per_stream);
+    un.n = min(max(p.n_keep[s], 0), p.keep_stride);
+    un.f = p.first_moved[s];
+    if (!p.in_place && un.f >= 0) un.f = 0;
+    const int total_chunks = un.f >= 0 && un.f < un.n ? (un.n - un.f + kChunkRows - 1) / kChunkRows : 0;
+    const int per_seg = max((total_chunks + split - 1) / split, 1);
+    un.n_seg = (total_chunks + per_seg - 1) / per_seg;  // non-empty segments
+    // invalid: keep list rejected, nothing moves, or fewer segments than `split`
+    un.valid = un.h < un.n_seg;
+    const int c_begin = un.h * per_seg, c_end = min(total_chunks, c_begin + per_seg);
+    un.j_begin = un.f + c_begin * kChunkRows;
+    un.j_end = min(un.n, un.f + c_end * kChunkRows);
+    un.seg_rows = per_seg * kChunkRows;
+    un.src = (tensor ? p.src[1] : p.src[0]) + (size_t)plane * p.capacity * p.row_bytes;
+    un.dst = (tensor ? p.dst[1] : p.dst[0]) + (size_t)plane * p.capacity * p.row_bytes;
+    un.keep = p.keep_idx + (size_t)s * p.keep_stride;
+    un.chained = p.in_place && un.n_seg > 1;
+    un.prog = p.plane_progress + (un.chained ? (size_t)r * kMaxSplit : 0);
+    return un;
+}
+
 // One warp waits (bounded) until the ready words of all n_streams streams are up.
 __device__ __forceinline__ bool wait_until_ready(const int32_t* ready, int n_streams, int lane) {
     int ok = 1;
@@ -217,63 +259,68 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
     __syncthreads();
     unsigned long long drawn = first_ticket == ~0ull ? ~0ull : first_ticket + wid;  // lane 0's copy counts
     alive = alive && drawn != ~0ull;
-    while (alive) {
-        const int64_t u = (int64_t)__shfl_sync(0xFFFFFFFFu, drawn, 0);
-        if (u >= n_units) break;
-        bool need_draw = true;  // the next number is drawn towards the end of this unit
-        auto draw = [&]() {
-            if (need_draw && lane == 0) drawn = atomicAdd(p.ticket, 1ull);
-            need_draw = false;
-        };
-        const int h = (int)(u / units_base);  // segment of the plane's moved rows
-        const int r = (int)(u - (int64_t)h * units_base);
-        const int tensor = (int)(r / p.planes_per_tensor);
-        const int64_t plane = r - (int64_t)tensor * p.planes_per_tensor;
-        const int s = (int)(plane / p.planes_per_stream);
-        const int n = min(max(p.n_keep[s], 0), p.keep_stride);
-        int f = p.first_moved[s];
-        if (!p.in_place && f >= 0) f = 0;
-        const int total_chunks = f >= 0 && f < n ? (n - f + kChunkRows - 1) / kChunkRows : 0;
-        const int per_seg = max((total_chunks + split - 1) / split, 1);
-        const int n_seg = (total_chunks + per_seg - 1) / per_seg;  // non-empty segments
-        if (h >= n_seg) {  // keep list rejected, nothing moves, or fewer segments than `split`
-            draw();
-            continue;
-        }
-        ++unit_no;  // counts the units that put chunks into the ring
-        const int c_begin = h * per_seg, c_end = min(total_chunks, c_begin + per_seg);
-        const int j_begin = f + c_begin * kChunkRows, j_end = min(n, f + c_end * kChunkRows);
 
-        const char* src = (tensor ? p.src[1] : p.src[0]) + (size_t)plane * p.capacity * p.row_bytes;
-        char* dst = (tensor ? p.dst[1] : p.dst[0]) + (size_t)plane * p.capacity * p.row_bytes;
-        const int32_t* keep = p.keep_idx + (size_t)s * p.keep_stride;
-        const bool chained = p.in_place && n_seg > 1;
-        if (chained && lane == 0) {
-            UnitInfo ui;
-            ui.keep = keep;
-            ui.prog = p.plane_progress + (size_t)r * kMaxSplit;
-            ui.seg = h;
-            ui.first = f;
-            ui.seg_rows = per_seg * kChunkRows;
-            ui.n = n;
-            units[unit_no % kMaxStages] = ui;
+    // the unit behind the number lane 0 holds; numbers whose unit is empty are skipped
+    auto next_unit = [&]() -> Unit {
+        Unit un;
+        un.valid = false;
+        while (alive) {
+            const int64_t u = (int64_t)__shfl_sync(0xFFFFFFFFu, drawn, 0);
+            if (u >= n_units) break;
+            un = resolve_unit(p, u, units_base, split);
+            if (un.valid) break;
+            if (lane == 0) drawn = atomicAdd(p.ticket, 1ull);
         }
-
-        // source rows of the next kIdxAhead chunks, one per lane and chunk, fetched a whole
-        // group ahead so that the index loads never sit on the critical path
-        int kq[kIdxAhead];
+        return un;
+    };
+    // source rows of a unit's first kIdxAhead chunks, one per lane and chunk
+    auto first_indices = [&](const Unit& un, int (&k)[kIdxAhead]) {
 #pragma unroll
         for (int q = 0; q < kIdxAhead; ++q) {
-            const int j = j_begin + q * kChunkRows + lane;
-            kq[q] = j < j_end ? keep[j] : -2;
+            const int j = un.j_begin + q * kChunkRows + lane;
+            k[q] = (un.valid && j < un.j_end) ? un.keep[j] : -2;
         }
+    };
+
+    // Source indices are always fetched a whole group of chunks ahead, across unit boundaries
+    // too: two groups before a unit ends the next number is drawn, one group before the end
+    // that unit is resolved and its first indices are requested, so that neither the counter
+    // nor the index loads sit on the critical path when the worker moves on.
+    Unit cur = next_unit();
+    int kq[kIdxAhead];
+    first_indices(cur, kq);
+    while (alive && cur.valid) {
+        ++unit_no;  // counts the units that put chunks into the ring
+        if (cur.chained && lane == 0) {
+            UnitInfo ui;
+            ui.keep = cur.keep;
+            ui.prog = cur.prog;
+            ui.seg = cur.h;
+            ui.first = cur.f;
+            ui.seg_rows = cur.seg_rows;
+            ui.n = cur.n;
+            units[unit_no % kMaxStages] = ui;
+        }
+        const int j_begin = cur.j_begin, j_end = cur.j_end;
+        bool drew = false, resolved = false;
+        Unit nxt;
+        nxt.valid = false;
+        int kq_next[kIdxAhead];
         for (int jg = j_begin; jg < j_end && alive; jg += kIdxAhead * kChunkRows) {
-            if (jg + 2 * kIdxAhead * kChunkRows >= j_end) draw();
+            if (!drew && jg + 2 * kIdxAhead * kChunkRows >= j_end) {
+                if (lane == 0) drawn = atomicAdd(p.ticket, 1ull);
+                drew = true;
+            }
+            if (!resolved && jg + kIdxAhead * kChunkRows >= j_end) {
+                nxt = next_unit();
+                first_indices(nxt, kq_next);
+                resolved = true;
+            }
             int kn[kIdxAhead];
 #pragma unroll
             for (int q = 0; q < kIdxAhead; ++q) {
                 const int j = jg + (kIdxAhead + q) * kChunkRows + lane;
-                kn[q] = j < j_end ? keep[j] : -2;
+                kn[q] = j < j_end ? cur.keep[j] : -2;
             }
 #pragma unroll
             for (int q = 0; q < kIdxAhead; ++q) {
@@ -285,12 +332,12 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
                 if (lane == 0) {
                     if (it >= stages) bulk_wait_read<kStoreSlack>();  // the stage's last store has left
                     StageInfo si;
-                    si.dst = dst + (size_t)j0 * p.row_bytes;
+                    si.dst = cur.dst + (size_t)j0 * p.row_bytes;
                     si.bytes = (uint32_t)nrows * p.row_bytes;
-                    si.d_end = (chained && h > 0) ? j0 + nrows : 0;
+                    si.d_end = (cur.chained && cur.h > 0) ? j0 + nrows : 0;
                     si.unit = unit_no;
                     const int done = (j0 - j_begin) / kChunkRows + 1;  // chunks of the segment so far
-                    si.publish = (chained && h + 1 < n_seg &&
+                    si.publish = (cur.chained && cur.h + 1 < cur.n_seg &&
                                   (done % kPublishEvery == 0 || j0 + kChunkRows >= j_end))
                                      ? (uint32_t)done
                                      : 0u;
@@ -306,7 +353,7 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
                     const uint32_t later = lane == 31 ? 0u : (heads & ~((2u << lane) - 1u));
                     const int next = later ? __ffs(later) - 1 : nrows;
                     bulk_load(buf + (size_t)stage * stage_bytes + (size_t)lane * p.row_bytes,
-                              src + (size_t)kj * p.row_bytes, (uint32_t)(next - lane) * p.row_bytes,
+                              cur.src + (size_t)kj * p.row_bytes, (uint32_t)(next - lane) * p.row_bytes,
                               &full[stage]);
                 }
                 ++it;
@@ -318,7 +365,9 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
 #pragma unroll
             for (int q = 0; q < kIdxAhead; ++q) kq[q] = kn[q];
         }
-        draw();
+        cur = nxt;
+#pragma unroll
+        for (int q = 0; q < kIdxAhead; ++q) kq[q] = kq_next[q];
     }
     while (alive && stored < it) {
         alive = store_chunk(full, info, units, buf, stored, stages, stage_bytes, lane, epoch, safe);
@@ -487,13 +536,11 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     if (units64 > 0x3FFFFFFF) return cudaErrorInvalidValue;
     const int units_base = (int)units64;
 
-    int dev = 0, n_sm = 0, smem_max = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    DeviceProps dp;
+    cudaError_t e = device_props(&dp);
     if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    if (e != cudaSuccess) return e;
+    const int n_sm = dp.n_sm, smem_max = dp.smem_optin;
+    static unsigned char allowed_ring[kMaxDevices], allowed_small[kMaxDevices];
 
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -510,8 +557,7 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
             col_splits *= 2;
         const size_t small_smem = (size_t)p.keep_stride * (p.row_bytes / col_splits);
         if (small_smem <= (size_t)smem_max - 1024) {
-            e = cudaFuncSetAttribute(compact_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)small_smem);
+            e = allow_max_dynamic_smem((const void*)compact_small_kernel, dp, allowed_small);
             if (e != cudaSuccess) return e;
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3((unsigned)(units_base * col_splits));
@@ -536,14 +582,24 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     if ((size_t)workers * stages * stage_bytes > budget) return cudaErrorInvalidValue;
     while (stages < 8 && (size_t)workers * (stages + 1) * stage_bytes <= budget) ++stages;
     const size_t smem = header_bytes(workers) + (size_t)workers * stages * stage_bytes;
-    e = cudaFuncSetAttribute(compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = allow_max_dynamic_smem((const void*)compact_kernel, dp, allowed_ring);
     if (e != cudaSuccess) return e;
 
     // a persistent grid: as many CTAs as the device keeps resident at once (the ring fills an
-    // SM's shared memory, so one per SM), fewer when there is less work
+    // SM's shared memory, so one per SM), fewer when there is less work.  The occupancy of a
+    // geometry is asked of the runtime once per device and remembered.
+    static std::atomic<long long> occ_cache[kMaxDevices];  // (smem << 20 | workers << 8 | per_sm) + 1
+    const long long occ_key = ((long long)smem << 20) | ((long long)workers << 8);
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compact_kernel, workers * 32, smem);
-    if (e != cudaSuccess) return e;
+    const bool slot = dp.device >= 0 && dp.device < kMaxDevices;
+    const long long seen = slot ? occ_cache[dp.device].load(std::memory_order_acquire) - 1 : -1;
+    if (seen >= 0 && (seen & ~0xFFll) == occ_key) {
+        per_sm = (int)(seen & 0xFF);
+    } else {
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compact_kernel, workers * 32, smem);
+        if (e != cudaSuccess) return e;
+        if (slot) occ_cache[dp.device].store((occ_key | (per_sm & 0xFF)) + 1, std::memory_order_release);
+    }
     if (per_sm < 1) return cudaErrorLaunchOutOfResources;
     const int64_t resident = (int64_t)n_sm * per_sm;
     // Cut planes into segments so that every worker draws a few dozen units: the ticket

@@ -130,9 +130,10 @@ cudaError_t launch_rerotate(const RopeParams& p, int n_streams, bool bf16, cudaS
     const int units = p.head_dim / 16;
     const int rows_per_block = kRopeThreads / units;
     const unsigned gx = (unsigned)((p.keep_stride + rows_per_block - 1) / rows_per_block);
-    int dev = 0, n_sm = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess)
-        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    DeviceProps dp;
+    cudaError_t e = device_props(&dp);
+    if (e != cudaSuccess) return e;
+    const int n_sm = dp.n_sm;
     // enough blocks to fill the GPU a few times over; each block reuses its angles over a group
     // of planes
     int64_t groups = ((int64_t)8 * n_sm + (int64_t)gx * n_streams - 1) / ((int64_t)gx * n_streams);

@@ -297,10 +297,10 @@ cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
     // 4 warps per CTA stream 16 KB each; a grid too small to give every SM even 8 warps takes
     // 8 or 16 warps per CTA instead (same bytes per CTA, shorter serial loop per warp).  With
     // more warps already resident, wider CTAs measured slower.
-    int dev = 0, n_sm = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess)
-        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    const int64_t want_warps = (int64_t)n_sm * 8;
+    DeviceProps dp;
+    cudaError_t e = device_props(&dp);
+    if (e != cudaSuccess) return e;
+    const int64_t want_warps = (int64_t)dp.n_sm * 8;
     const int warps = ctas * 4 >= want_warps ? 4 : (ctas * 8 >= want_warps ? 8 : 16);
     const bool bf16 = p.logits_dtype == SIRLLM_BF16;
     if (warps == 4) {

@@ -375,15 +375,14 @@ cudaError_t launch_select(const SelectParams& p, int n_streams, cudaStream_t st,
     // scores (rounded up to whole 128-bit vectors, plus one vector of slack) + histogram
     // (+ the staged keep list when it fits)
     size_t smem = ((size_t)((p.capacity + 3) & ~3) + 4) * 4 + (size_t)kRadixBins * 4;
-    int dev = 0, smem_max = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    DeviceProps dp;
+    cudaError_t e = device_props(&dp);
     if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    if (e != cudaSuccess) return e;
-    const bool stage = smem + (size_t)p.threshold * 4 + 1024 <= (size_t)smem_max;
+    const bool stage = smem + (size_t)p.threshold * 4 + 1024 <= (size_t)dp.smem_optin;
     if (stage) smem += (size_t)p.threshold * 4;
+    static unsigned char allowed[2][kMaxDevices];
     auto kernel = stage ? select_kernel<true> : select_kernel<false>;
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = allow_max_dynamic_smem((const void*)kernel, dp, allowed[stage ? 1 : 0]);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)n_streams);

@@ -824,3 +824,27 @@ def test_a_device_side_wait_that_runs_out_is_reported_not_hung():
     assert B.sirllm_status(st.ws) == 0
     st.check_kv_by_content()
     assert st.host_len == [64]
+
+
+def test_prepared_call_repeats_the_checked_call():
+    # arguments are checked and marshalled once; every later invocation issues the same call on
+    # whatever the tensors hold by then
+    w = wl.WORKLOADS["tiny"].scaled(n_layers=1, n_kv_heads=2, capacity=256, budget=96, n_recent=16,
+                                    new_tokens=70, vocab=3001)
+    a, b = DeviceState(w), DeviceState(w)
+    step = B.prepared(B.sirllm_step, b.cfg, b.logits, b.token_ids, b.n_new, b.scores, b.serial, b.live_len,
+                      b.decay, b.k, b.v, b.keep_idx, b.n_keep, b.new_entropy, b.ws)
+    for r in range(4):
+        a.fill_round(r)
+        b.fill_round(r)
+        a.step()
+        step()
+        b.host_len = b.live_len.cpu().tolist()
+        assert a.host_len == b.host_len
+        n = a.host_len[0]
+        assert torch.equal(a.keep_idx[:, :n], b.keep_idx[:, :n])
+        assert torch.equal(a.scores[:, :n].view(torch.int32), b.scores[:, :n].view(torch.int32))
+        assert torch.equal(a.k[:, :, :n], b.k[:, :, :n]) and torch.equal(a.v[:, :, :n], b.v[:, :, :n])
+    with pytest.raises(B.SirllmError):                       # the checks still run, once
+        B.prepared(B.sirllm_step, b.cfg, b.logits, b.token_ids[:5], b.n_new, b.scores, b.serial, b.live_len,
+                   b.decay, b.k, b.v, b.keep_idx, b.n_keep, b.new_entropy, b.ws)
