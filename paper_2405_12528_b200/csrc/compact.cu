@@ -15,7 +15,7 @@
 // chunk is stored only after its loads and those of all earlier chunks of the plane have
 // landed, and later chunks only read rows behind everything stored so far.
 //
-// To fill all SMs evenly, the moved rows of a plane are cut into `split` segments that
+// To fill all SMs evenly, the moved rows of a plane are cut into segments of `seg_chunks` chunks that
 // different workers take.  Work units (plane, segment) are numbered segment-major, so a
 // plane's earlier segments come long before its later ones, and are handed out in that order
 // through one ticket counter in the workspace: a worker that is about to run dry draws the
@@ -50,7 +50,8 @@ constexpr int kIdxAhead = 4;     // chunks whose source indices are fetched ahea
 constexpr int kMaxWorkers = 4;   // worker warps per CTA
 constexpr int kPublishEvery = 4; // chunks between two updates of a segment's progress word
 constexpr int kNoBound = 0x7FFFFFFF;
-constexpr int kUnitsPerWorker = 28;  // work units per worker the split of the planes aims at
+constexpr int kUnitsPerWorker = 34;  // work units per worker the split of the planes aims at
+constexpr int kMinSegChunks = 5;     // shortest segment (chunks) worth a unit's set-up
 constexpr int64_t kSmallJobBytes = 8 << 20;  // planes x longest keep list x row: the two-phase kernel's range
 
 // What the store of a chunk needs to know about the chunk ...
@@ -161,7 +162,7 @@ struct Unit {
     bool valid;                // false: nothing to move for this number
 };
 
-__device__ __forceinline__ Unit resolve_unit(const CompactParams& p, int64_t u, int units_base, int split) {
+__device__ __forceinline__ Unit resolve_unit(const CompactParams& p, int64_t u, int units_base, int seg_chunks) {
     Unit un;
     un.h = (int)(u / units_base);  // segment of the plane's moved rows
     const int r = (int)(u - (int64_t)un.h * units_base);
@@ -172,9 +173,9 @@ __device__ __forceinline__ Unit resolve_unit(const CompactParams& p, int64_t u, 
     un.f = p.first_moved[s];
     if (!p.in_place && un.f >= 0) un.f = 0;
     const int total_chunks = un.f >= 0 && un.f < un.n ? (un.n - un.f + kChunkRows - 1) / kChunkRows : 0;
-    const int per_seg = max((total_chunks + split - 1) / split, 1);
+    const int per_seg = seg_chunks;
     un.n_seg = (total_chunks + per_seg - 1) / per_seg;  // non-empty segments
-    // invalid: keep list rejected, nothing moves, or fewer segments than `split`
+    // invalid: keep list rejected, nothing moves, or a segment behind the stream's last one
     un.valid = un.h < un.n_seg;
     const int c_begin = un.h * per_seg, c_end = min(total_chunks, c_begin + per_seg);
     un.j_begin = un.f + c_begin * kChunkRows;
@@ -212,7 +213,8 @@ __host__ __device__ inline size_t header_bytes(int n_workers) {
 }
 
 __global__ void __launch_bounds__(kMaxWorkers * 32, 1)
-compact_kernel(const CompactParams p, const int stages, const int units_base, const int split) {
+compact_kernel(const CompactParams p, const int stages, const int units_base, const int split,
+               const int seg_chunks) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int n_workers = blockDim.x >> 5;
     const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -267,7 +269,7 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
         while (alive) {
             const int64_t u = (int64_t)__shfl_sync(0xFFFFFFFFu, drawn, 0);
             if (u >= n_units) break;
-            un = resolve_unit(p, u, units_base, split);
+            un = resolve_unit(p, u, units_base, seg_chunks);
             if (un.valid) break;
             if (lane == 0) drawn = atomicAdd(p.ticket, 1ull);
         }
@@ -604,17 +606,25 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     const int64_t resident = (int64_t)n_sm * per_sm;
     // Cut planes into segments so that every worker draws a few dozen units: the ticket
     // hand-out then evens out SMs of different speed down to a small tail, while a unit stays
-    // long enough (at least four chunks at the longest keep list) to amortise its set-up.
-    // About 28 units per worker measured best on every shape tried (14 and 55 were worse).
+    // long enough to amortise its set-up.  Segments are a fixed number of chunks long
+    // (`seg_chunks`), chosen ODD: planes are a power of two apart, so segments of 2^k chunks
+    // would make all workers walk addresses that differ by large powers of two at the same
+    // time, which measured 2-3 % slower than odd lengths around the same size.  Around 34 units
+    // per worker measured best over the shapes tried (20 to 40 are within a percent; 14 and 55
+    // are worse).
     const int64_t slots = resident * workers;
-    int split = 1;
+    const int64_t chunks_max = (p.keep_stride + kChunkRows - 1) / kChunkRows;
+    int64_t seg_chunks = chunks_max;  // one segment per plane
     if (units_base <= kChainPlanesMax) {
-        const int64_t chunks_max = (p.keep_stride + kChunkRows - 1) / kChunkRows;
-        int64_t want_split = (kUnitsPerWorker * slots + units_base / 2) / units_base;
-        if (want_split > chunks_max / 4) want_split = chunks_max / 4;
-        if (want_split > kMaxSplit) want_split = kMaxSplit;
-        if (want_split > 1) split = (int)want_split;
+        // chunks of all planes shared out over kUnitsPerWorker units per worker
+        int64_t want = (chunks_max * units_base + kUnitsPerWorker * slots / 2) / (kUnitsPerWorker * slots);
+        if (want < kMinSegChunks) want = kMinSegChunks;
+        if (want % 2 == 0) ++want;
+        const int64_t least = (chunks_max + kMaxSplit - 1) / kMaxSplit;  // at most kMaxSplit segments
+        if (want < least) want = least;
+        if (want < chunks_max) seg_chunks = want;
     }
+    const int split = (int)((chunks_max + seg_chunks - 1) / seg_chunks);
     const int64_t n_units = (int64_t)units_base * split;
     const int64_t want = (n_units + workers - 1) / workers;
     const int grid = (int)(want < resident ? want : resident);
@@ -625,7 +635,7 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, compact_kernel, q, stages, units_base, split);
+    return cudaLaunchKernelEx(&cfg, compact_kernel, q, stages, units_base, split, (int)seg_chunks);
 }
 
 }  // namespace sirllm

@@ -10,9 +10,8 @@
 // group; per plane it moves two 16-byte vectors.  The rotation itself is also carried out in
 // fp64 and every element is rounded ONCE, from fp64, to bf16/fp16: the result is the exactly
 // rotated value rounded to nearest even (an fp32 rotation loses the low bits of the products
-// where x cos - y sin cancels).  The rounding to the 16-bit precision is done by the fp64 adder
-// (add and subtract a power of two chosen from the value's exponent), after which the
-// narrowing conversions are exact.
+// where x cos - y sin cancels).  Widening to fp64 and the rounding back are done with integer
+// operations on the bit patterns, so the arithmetic stays under the memory time.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -24,26 +23,56 @@ namespace {
 
 constexpr int kRopeThreads = 128;
 
+// Layout constants of the two storage types inside an fp64 bit pattern: a normal 16-bit value
+// is its magnitude bits shifted up by kShift inside the double's high word with the exponent
+// re-biased by kBias (1023 - 127 for bf16, 1023 - 15 for fp16).
+template <bool kBf16>
+struct Fmt {
+    static constexpr int kShift = kBf16 ? 13 : 10;             // high-word bits below the 16-bit mantissa
+    static constexpr uint32_t kBias = kBf16 ? 896u : 1008u;
+    static constexpr uint32_t kExpMask = kBf16 ? 0x7F80u : 0x7C00u;
+    static constexpr uint32_t kExpMax = kBf16 ? 255u : 31u;    // exponent field of inf / nan
+    static constexpr int kExpPos = kBf16 ? 7 : 10;             // position of the exponent field
+};
+
+// 16-bit element -> fp64, exactly.  Normal values and zeros are widened with integer operations
+// (conversions to and from fp64 are a quarter-rate pipe and would bound the kernel); subnormals,
+// infinities and nans take the conversion instructions.
 template <bool kBf16>
 __device__ __forceinline__ double load16(uint32_t word, int hi) {
-    const uint16_t h = hi ? (uint16_t)(word >> 16) : (uint16_t)(word & 0xFFFFu);
-    if (kBf16) return (double)__uint_as_float((uint32_t)h << 16);
-    return (double)__half2float(__ushort_as_half(h));
+    using F = Fmt<kBf16>;
+    const uint32_t h = hi ? word >> 16 : word & 0xFFFFu;
+    const uint32_t mag = h & 0x7FFFu, ex = mag & F::kExpMask, sign = (h & 0x8000u) << 16;
+    if (ex != 0 && ex != F::kExpMask)
+        return __hiloint2double((int)(sign | ((mag << F::kShift) + (F::kBias << 20))), 0);
+    if (mag == 0) return __hiloint2double((int)sign, 0);
+    if (kBf16) return (double)__uint_as_float(h << 16);
+    return (double)__half2float(__ushort_as_half((unsigned short)h));
 }
 
 // fp64 -> bit pattern of the nearest bf16 / fp16 value (ties to even), in one rounding.
-// With E the exponent of v, adding and subtracting 2^(E + 53 - p) (same sign as v) leaves v
-// rounded to p significant bits by the adder; E is clamped at the type's smallest normal
-// exponent so that subnormal results keep the subnormal spacing.  The rounded value is exact
-// in fp32 and in the 16-bit type.
+// Results in the type's normal range are rounded on the bit pattern: the bits below the 16-bit
+// mantissa are the low kShift bits of the high word and the whole low word, which only counts as
+// "something below" (folded into bit 0); adding half-minus-one plus the kept mantissa's last bit
+// carries into the kept part exactly when round-to-nearest-even rounds up, exponent included.
+// Everything else (subnormal results, overflow, nan) goes through the fp64 adder: with E the
+// exponent of v clamped at the smallest normal exponent, adding and subtracting 2^(E + 53 - p)
+// leaves v rounded to p significant bits, exact in fp32 and in the 16-bit type.
 template <bool kBf16>
 __device__ __forceinline__ uint32_t round16(double v) {
+    using F = Fmt<kBf16>;
+    const uint32_t hi = (uint32_t)__double2hiint(v), lo = (uint32_t)__double2loint(v);
+    const uint32_t mag = hi & 0x7FFFFFFFu, sign16 = (hi >> 16) & 0x8000u;
+    const uint32_t t = (mag | (lo != 0u ? 1u : 0u)) + ((1u << (F::kShift - 1)) - 1u) + ((mag >> F::kShift) & 1u);
+    const uint32_t ex = t >> 20;  // exponent after rounding (a carry may have raised it)
+    if (ex > F::kBias && ex < F::kBias + F::kExpMax)
+        return ((t >> F::kShift) - (F::kBias << F::kExpPos)) | sign16;
+    if ((mag | lo) == 0u) return sign16;  // keeps the sign of a zero
     constexpr int p = kBf16 ? 8 : 11, emin = kBf16 ? -126 : -14;
-    const int hi = __double2hiint(v);
-    const int e = max(hi & 0x7FF00000, (emin + 1023) << 20);
+    const int e = max((int)(hi & 0x7FF00000u), (emin + 1023) << 20);
     double r = v;
     if (e < 0x7FF00000) {  // finite
-        const double big = __hiloint2double((hi & (int)0x80000000) | (e + ((53 - p) << 20)), 0);
+        const double big = __hiloint2double((int)(hi & 0x80000000u) | (e + ((53 - p) << 20)), 0);
         r = __dsub_rn(__dadd_rn(v, big), big);
     }
     const float f = __double2float_rn(r);  // exact (or inf / nan)
@@ -52,7 +81,7 @@ __device__ __forceinline__ uint32_t round16(double v) {
         bits = __float_as_uint(f) >> 16;
     else
         bits = (uint32_t)__half_as_ushort(__float2half_rn(f));
-    return (bits & 0x7FFFu) | (((uint32_t)hi >> 16) & 0x8000u);  // keeps the sign of a zero
+    return (bits & 0x7FFFu) | sign16;
 }
 template <bool kBf16>
 __device__ __forceinline__ uint32_t pack16(double lo, double hi) {
