@@ -238,15 +238,13 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
     __syncwarp();
 
     // The kernel that precedes this one on the stream (selection, or the check of a caller's
-    // keep lists) raises ready[s] as soon as stream s's keep list and counts - and, with stream
-    // 0, the epoch and the ticket counter - are out, possibly long before it ends.  Under a
-    // programmatic dependent launch this grid polls those words instead of waiting for the whole
-    // preceding grid, so the gather starts while that kernel finishes its other work.  Every
-    // stream's word is awaited before anything that kernel wrote is read (lane i takes streams
-    // i, i + 32, ...), so those reads may go through L1.
-    bool alive = wait_until_ready(p.ready, (int)(p.planes_per_tensor / p.planes_per_stream), lane);
-
-    const uint32_t epoch = alive ? (uint32_t)*p.epoch : 0u;
+    // keep lists) sets the epoch and the ticket counter before this grid can start, and raises
+    // ready[s] as soon as stream s's keep list and counts are out, possibly long before it ends.
+    // Under a programmatic dependent launch this grid polls those words instead of waiting for
+    // the whole preceding grid, so the gather starts while that kernel finishes its other work.
+    // Every stream's word is awaited before anything else that kernel wrote is read (lane i
+    // takes streams i, i + 32, ...), so those reads may go through L1.
+    const uint32_t epoch = (uint32_t)*p.epoch;
     const int lead = stages - 1 - kStoreSlack;  // chunks whose loads run ahead of the stores
     const int64_t n_units = (int64_t)units_base * split;
     int64_t it = 0;      // chunks whose loads were issued
@@ -257,10 +255,10 @@ compact_kernel(const CompactParams p, const int stages, const int units_base, co
     // The first numbers are drawn once per CTA for all its workers (a quarter of the counter
     // traffic while the whole grid starts at once), later ones by each worker for itself.
     __shared__ unsigned long long first_ticket;
-    if (threadIdx.x == 0) first_ticket = alive ? atomicAdd(p.ticket, (unsigned long long)n_workers) : ~0ull;
+    if (threadIdx.x == 0) first_ticket = atomicAdd(p.ticket, (unsigned long long)n_workers);
+    bool alive = wait_until_ready(p.ready, (int)(p.planes_per_tensor / p.planes_per_stream), lane);
     __syncthreads();
-    unsigned long long drawn = first_ticket == ~0ull ? ~0ull : first_ticket + wid;  // lane 0's copy counts
-    alive = alive && drawn != ~0ull;
+    unsigned long long drawn = first_ticket + wid;  // lane 0's copy counts
 
     // the unit behind the number lane 0 holds; numbers whose unit is empty are skipped
     auto next_unit = [&]() -> Unit {
@@ -465,12 +463,17 @@ __global__ void compact_plan_kernel(const CompactParams p, int32_t* __restrict__
     if (threadIdx.x == 0) {
         sh_first = n;
         sh_bad = (p.n_keep[s] < 0 || p.n_keep[s] > p.keep_stride) ? 1 : 0;
-        if (s == 0) {  // a new compaction follows
+        // the same hand-off as the selection kernel's: ready word down, epoch and ticket counter
+        // set for the gather, all of it visible before the gather's grid may start
+        st_relaxed_u32(&p.ready[s], 0u);
+        if (s == 0) {
             *p.epoch += 1;
             *p.ticket = 0ull;
         }
+        __threadfence();
     }
     __syncthreads();
+    grid_launch_dependents();
     for (int j = threadIdx.x; j < n; j += blockDim.x) {
         const int kj = keep[j];
         const int prev = j > 0 ? keep[j - 1] : -1;

@@ -10,8 +10,9 @@
 // group; per plane it moves two 16-byte vectors.  The rotation itself is also carried out in
 // fp64 and every element is rounded ONCE, from fp64, to bf16/fp16: the result is the exactly
 // rotated value rounded to nearest even (an fp32 rotation loses the low bits of the products
-// where x cos - y sin cancels).  Widening to fp64 and the rounding back are done with integer
-// operations on the bit patterns, so the arithmetic stays under the memory time.
+// where x cos - y sin cancels).  The single rounding is obtained by truncating to fp32 with a
+// sticky last bit and letting the packed fp32 -> 16-bit conversion round (a few instructions per
+// element); the vectors of the next two planes are in flight while one plane is turned.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -23,69 +24,44 @@ namespace {
 
 constexpr int kRopeThreads = 128;
 
-// Layout constants of the two storage types inside an fp64 bit pattern: a normal 16-bit value
-// is its magnitude bits shifted up by kShift inside the double's high word with the exponent
-// re-biased by kBias (1023 - 127 for bf16, 1023 - 15 for fp16).
-template <bool kBf16>
-struct Fmt {
-    static constexpr int kShift = kBf16 ? 13 : 10;             // high-word bits below the 16-bit mantissa
-    static constexpr uint32_t kBias = kBf16 ? 896u : 1008u;
-    static constexpr uint32_t kExpMask = kBf16 ? 0x7F80u : 0x7C00u;
-    static constexpr uint32_t kExpMax = kBf16 ? 255u : 31u;    // exponent field of inf / nan
-    static constexpr int kExpPos = kBf16 ? 7 : 10;             // position of the exponent field
-};
-
-// 16-bit element -> fp64, exactly.  Normal values and zeros are widened with integer operations
-// (conversions to and from fp64 are a quarter-rate pipe and would bound the kernel); subnormals,
-// infinities and nans take the conversion instructions.
+// 16-bit element -> fp64, exactly (two conversions; bf16 -> fp32 is a shift).
 template <bool kBf16>
 __device__ __forceinline__ double load16(uint32_t word, int hi) {
-    using F = Fmt<kBf16>;
-    const uint32_t h = hi ? word >> 16 : word & 0xFFFFu;
-    const uint32_t mag = h & 0x7FFFu, ex = mag & F::kExpMask, sign = (h & 0x8000u) << 16;
-    if (ex != 0 && ex != F::kExpMask)
-        return __hiloint2double((int)(sign | ((mag << F::kShift) + (F::kBias << 20))), 0);
-    if (mag == 0) return __hiloint2double((int)sign, 0);
-    if (kBf16) return (double)__uint_as_float(h << 16);
-    return (double)__half2float(__ushort_as_half((unsigned short)h));
+    if (kBf16) return (double)__uint_as_float(hi ? word & 0xFFFF0000u : word << 16);
+    return (double)__half2float(__ushort_as_half((unsigned short)(hi ? word >> 16 : word & 0xFFFFu)));
 }
 
-// fp64 -> bit pattern of the nearest bf16 / fp16 value (ties to even), in one rounding.
-// Results in the type's normal range are rounded on the bit pattern: the bits below the 16-bit
-// mantissa are the low kShift bits of the high word and the whole low word, which only counts as
-// "something below" (folded into bit 0); adding half-minus-one plus the kept mantissa's last bit
-// carries into the kept part exactly when round-to-nearest-even rounds up, exponent included.
-// Everything else (subnormal results, overflow, nan) goes through the fp64 adder: with E the
-// exponent of v clamped at the smallest normal exponent, adding and subtracting 2^(E + 53 - p)
-// leaves v rounded to p significant bits, exact in fp32 and in the 16-bit type.
+// fp64 -> an fp32 value whose round-to-nearest-even conversion to bf16 / fp16 equals the
+// direct, single rounding of the fp64 value: "round to odd".  The fp64 value is truncated to
+// fp32 and, if any of the 29 mantissa bits that fp32 cannot hold was set, the last bit of the
+// fp32 mantissa is forced to one; fp32 keeps at least two bits more than either 16-bit type, so
+// the sticky last bit decides ties and near-ties exactly as the discarded bits would.
+// Values below the smallest normal fp32 (possible for bf16 when a rotation cancels almost
+// completely) lose more than 29 bits in the truncation; they are rounded to the type's
+// precision by the fp64 adder instead (add and subtract 2^(E + 53 - p), E clamped at the type's
+// smallest normal exponent), which leaves a value that is exact in fp32 and in the 16-bit type.
 template <bool kBf16>
-__device__ __forceinline__ uint32_t round16(double v) {
-    using F = Fmt<kBf16>;
+__device__ __forceinline__ float to_odd(double v) {
     const uint32_t hi = (uint32_t)__double2hiint(v), lo = (uint32_t)__double2loint(v);
-    const uint32_t mag = hi & 0x7FFFFFFFu, sign16 = (hi >> 16) & 0x8000u;
-    const uint32_t t = (mag | (lo != 0u ? 1u : 0u)) + ((1u << (F::kShift - 1)) - 1u) + ((mag >> F::kShift) & 1u);
-    const uint32_t ex = t >> 20;  // exponent after rounding (a carry may have raised it)
-    if (ex > F::kBias && ex < F::kBias + F::kExpMax)
-        return ((t >> F::kShift) - (F::kBias << F::kExpPos)) | sign16;
-    if ((mag | lo) == 0u) return sign16;  // keeps the sign of a zero
-    constexpr int p = kBf16 ? 8 : 11, emin = kBf16 ? -126 : -14;
-    const int e = max((int)(hi & 0x7FF00000u), (emin + 1023) << 20);
-    double r = v;
-    if (e < 0x7FF00000) {  // finite
-        const double big = __hiloint2double((int)(hi & 0x80000000u) | (e + ((53 - p) << 20)), 0);
-        r = __dsub_rn(__dadd_rn(v, big), big);
+    const uint32_t mag = hi & 0x7FFFFFFFu;
+    if (kBf16 && mag < 0x38100000u && (mag | lo) != 0u) {  // 0 < |v| < 2^-126
+        const double big = __hiloint2double((int)((hi & 0x80000000u) | ((uint32_t)(-126 + 1023 + 53 - 8) << 20)), 0);
+        return __double2float_rn(__dsub_rn(__dadd_rn(v, big), big));
     }
-    const float f = __double2float_rn(r);  // exact (or inf / nan)
-    uint32_t bits;
-    if (kBf16)
-        bits = __float_as_uint(f) >> 16;
-    else
-        bits = (uint32_t)__half_as_ushort(__float2half_rn(f));
-    return (bits & 0x7FFFu) | sign16;
+    float f = __double2float_rz(v);
+    if ((lo & 0x1FFFFFFFu) != 0u) f = __uint_as_float(__float_as_uint(f) | 1u);
+    return f;
 }
+// two fp64 values -> one word of two 16-bit elements (first argument in the low half)
 template <bool kBf16>
 __device__ __forceinline__ uint32_t pack16(double lo, double hi) {
-    return round16<kBf16>(lo) | (round16<kBf16>(hi) << 16);
+    const float f0 = to_odd<kBf16>(lo), f1 = to_odd<kBf16>(hi);
+    uint32_t out;
+    if (kBf16)
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out) : "f"(f1), "f"(f0));
+    else
+        asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(out) : "f"(f1), "f"(f0));
+    return out;
 }
 // one pair turned by the angle whose cosine and sine are c and s: each product and each sum is
 // a separately rounded fp64 operation
@@ -119,37 +95,56 @@ __global__ void __launch_bounds__(kRopeThreads) rerotate_kernel(const RopeParams
     const size_t row_bytes = (size_t)p.head_dim * 2;
     const int pl0 = blockIdx.z * p.planes_per_group;
     const int pl1 = min(p.planes_per_stream, pl0 + p.planes_per_group);
-    for (int pl = pl0; pl < pl1; ++pl) {
-        char* row = p.k + (((size_t)s * p.planes_per_stream + pl) * p.capacity + j) * row_bytes;
-        uint4* pa = reinterpret_cast<uint4*>(row + (p.layout == SIRLLM_ROPE_HALF ? 16 * u : 32 * u));
-        uint4* pb = reinterpret_cast<uint4*>(
-            row + (p.layout == SIRLLM_ROPE_HALF ? (size_t)p.head_dim + 16 * u : 32 * u + 16));
-        const uint4 a = *pa, b = *pb;
-        const uint32_t wa[4] = {a.x, a.y, a.z, a.w}, wb[4] = {b.x, b.y, b.z, b.w};
-        uint32_t oa[4], ob[4];
-        if (p.layout == SIRLLM_ROPE_HALF) {  // a holds x of pairs 8u..8u+7, b holds their y
+    const size_t plane_stride = (size_t)p.capacity * row_bytes;
+    char* row0 = p.k + (((size_t)s * p.planes_per_stream + pl0) * p.capacity + j) * row_bytes;
+    const size_t off_a = p.layout == SIRLLM_ROPE_HALF ? 16 * u : 32 * u;
+    const size_t off_b = p.layout == SIRLLM_ROPE_HALF ? (size_t)p.head_dim + 16 * u : 32 * u + 16;
+    constexpr int kAhead = 2;  // planes whose vectors are in flight while one is turned
+    uint4 qa[kAhead], qb[kAhead];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                double x[2], y[2];
-#pragma unroll
-                for (int h = 0; h < 2; ++h)
-                    turn(load16<kBf16>(wa[q], h), load16<kBf16>(wb[q], h), cs[2 * q + h],
-                         sn[2 * q + h], x[h], y[h]);
-                oa[q] = pack16<kBf16>(x[0], x[1]);
-                ob[q] = pack16<kBf16>(y[0], y[1]);
-            }
-        } else {  // every 32-bit word is one pair (x, y): a = pairs 8u..8u+3, b = 8u+4..8u+7
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                double xo, yo;
-                turn(load16<kBf16>(wa[q], 0), load16<kBf16>(wa[q], 1), cs[q], sn[q], xo, yo);
-                oa[q] = pack16<kBf16>(xo, yo);
-                turn(load16<kBf16>(wb[q], 0), load16<kBf16>(wb[q], 1), cs[4 + q], sn[4 + q], xo, yo);
-                ob[q] = pack16<kBf16>(xo, yo);
-            }
+    for (int d = 0; d < kAhead; ++d) {
+        if (pl0 + d < pl1) {
+            qa[d] = *reinterpret_cast<const uint4*>(row0 + d * plane_stride + off_a);
+            qb[d] = *reinterpret_cast<const uint4*>(row0 + d * plane_stride + off_b);
         }
-        *pa = make_uint4(oa[0], oa[1], oa[2], oa[3]);
-        *pb = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+    }
+    for (int base = pl0; base < pl1; base += kAhead) {
+#pragma unroll
+        for (int d = 0; d < kAhead; ++d) {
+            const int pl = base + d;
+            if (pl >= pl1) break;
+            char* row = row0 + (size_t)(pl - pl0) * plane_stride;
+            const uint4 a = qa[d], b = qb[d];
+            if (pl + kAhead < pl1) {  // the plane that takes this buffer next
+                qa[d] = *reinterpret_cast<const uint4*>(row + kAhead * plane_stride + off_a);
+                qb[d] = *reinterpret_cast<const uint4*>(row + kAhead * plane_stride + off_b);
+            }
+            const uint32_t wa[4] = {a.x, a.y, a.z, a.w}, wb[4] = {b.x, b.y, b.z, b.w};
+            uint32_t oa[4], ob[4];
+            if (p.layout == SIRLLM_ROPE_HALF) {  // a holds x of pairs 8u..8u+7, b holds their y
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    double x[2], y[2];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        turn(load16<kBf16>(wa[q], h), load16<kBf16>(wb[q], h), cs[2 * q + h],
+                             sn[2 * q + h], x[h], y[h]);
+                    oa[q] = pack16<kBf16>(x[0], x[1]);
+                    ob[q] = pack16<kBf16>(y[0], y[1]);
+                }
+            } else {  // every 32-bit word is one pair (x, y): a = pairs 8u..8u+3, b = 8u+4..8u+7
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    double xo, yo;
+                    turn(load16<kBf16>(wa[q], 0), load16<kBf16>(wa[q], 1), cs[q], sn[q], xo, yo);
+                    oa[q] = pack16<kBf16>(xo, yo);
+                    turn(load16<kBf16>(wb[q], 0), load16<kBf16>(wb[q], 1), cs[4 + q], sn[4 + q], xo, yo);
+                    ob[q] = pack16<kBf16>(xo, yo);
+                }
+            }
+            *reinterpret_cast<uint4*>(row + off_a) = make_uint4(oa[0], oa[1], oa[2], oa[3]);
+            *reinterpret_cast<uint4*>(row + off_b) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+        }
     }
 }
 

@@ -95,9 +95,15 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     const int cap = p.capacity;
     float* scores = p.scores + (size_t)s * cap;
     int32_t* keep = p.keep_idx + (size_t)s * p.threshold;
-    // the gather polls ready[s]: take it down before any dependent grid can start
+    // the gather polls ready[s]: take it down before any dependent grid can start; with it the
+    // gather's epoch and ticket counter are set for the compaction that follows (everything
+    // earlier on the stream, the previous gather included, is complete when this grid starts)
     if (tid == 0) {
         st_relaxed_u32(&p.ready[s], 0u);
+        if (blockIdx.x == 0) {
+            *p.epoch += 1;
+            *p.ticket = 0ull;
+        }
         __threadfence();
     }
     __syncthreads();
@@ -116,13 +122,7 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
     }
     if (l0 < 0 || l0 > cap - T) {  // the round does not fit: leave the stream alone
         grid_dependency_wait();
-        if (tid == 0) {
-            if (blockIdx.x == 0) {
-                *p.epoch += 1;
-                *p.ticket = 0ull;
-            }
-            atomicOr(p.status, SIRLLM_STATUS_OVERFLOW);
-        }
+        if (tid == 0) atomicOr(p.status, SIRLLM_STATUS_OVERFLOW);
         const int n = max(0, min(l0, min(cap, p.threshold)));
         publish_keep_list(p, s, n, n);  // nothing moves
         return;
@@ -162,11 +162,8 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
         }
     };
     decay_range(0, l0);      // the scores of earlier rounds
+    for (int b = tid; b < kRadixBins; b += kSelectThreads) hist[b] = 0;  // for the first digit pass
     grid_dependency_wait();  // the scorer's appended scores are complete and visible
-    if (blockIdx.x == 0 && tid == 0) {  // a new compaction follows
-        *p.epoch += 1;
-        *p.ticket = 0ull;
-    }
     decay_range(l0, l);      // this round's scores
     if (!evict) {  // ---- nothing to evict: identity keep list --------------------------
         for (int i = tid; i < l; i += kSelectThreads) keep[i] = i;
@@ -202,11 +199,15 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
         int undecided = range ? 32 - __clz(range) : 0;  // low bits of d not yet fixed
         uint32_t prefix = 0u;                           // the fixed high bits of d
         int need = k;
+        bool first_pass = true;  // its histogram was zeroed ahead of the wait
         while (undecided > 0) {
             const int w = min(kRadixBits, undecided);
             const int sh_amt = undecided - w;
-            for (int b = tid; b < kRadixBins; b += kSelectThreads) hist[b] = 0;
-            __syncthreads();
+            if (!first_pass) {
+                for (int b = tid; b < kRadixBins; b += kSelectThreads) hist[b] = 0;
+                __syncthreads();
+            }
+            first_pass = false;
             for (int i = lo + tid; i < hi; i += kSelectThreads) {
                 const uint32_t d = order_key(vals[i]) - kmin;
                 if ((uint32_t)((uint64_t)d >> undecided) == prefix)
@@ -244,16 +245,25 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
                     if ((d >> undecided) == prefix) list[atomicAdd(&sh.list_n, 1)] = d;
                 }
                 __syncthreads();
-                if (tid < n_left) {
-                    const uint32_t mine = list[tid];
+                {
+                    // a team of four threads ranks one listed key, each against a quarter of the list
+                    static_assert(kListMax * 4 == kSelectThreads, "one team of four per listed key");
+                    const int e = tid >> 2, part = tid & 3;
+                    const uint32_t mine = e < n_left ? list[e] : 0u;
                     int greater = 0, equal = 0;
-                    for (int j = 0; j < n_left; ++j) {
-                        const uint32_t other = list[j];
-                        greater += other > mine;
-                        equal += other == mine;
+                    if (e < n_left) {
+                        for (int j = part; j < n_left; j += 4) {
+                            const uint32_t other = list[j];
+                            greater += other > mine;
+                            equal += other == mine;
+                        }
                     }
-                    if (greater < need && need <= greater + equal) {  // the need-th largest
-                        sh.tau = mine;
+                    greater += __shfl_xor_sync(0xFFFFFFFFu, greater, 1);
+                    equal += __shfl_xor_sync(0xFFFFFFFFu, equal, 1);
+                    greater += __shfl_xor_sync(0xFFFFFFFFu, greater, 2);
+                    equal += __shfl_xor_sync(0xFFFFFFFFu, equal, 2);
+                    if (e < n_left && part == 0 && greater < need && need <= greater + equal) {
+                        sh.tau = mine;  // the need-th largest
                         sh.r = need - greater;
                     }
                 }
