@@ -12,7 +12,10 @@
  *     The library allocates nothing and keeps no device state between calls; the
  *     caller owns every buffer, including the workspace `ws`
  *     (sirllm_workspace_bytes() bytes, 256-byte aligned, set up once with
- *     sirllm_workspace_init()).
+ *     sirllm_workspace_init()).  On the host it remembers, per device, a few properties
+ *     it would otherwise ask the runtime for at every call (SM count, shared-memory
+ *     limit, the occupancy of its gather kernel).  Launches carry NVTX ranges
+ *     ("sirllm:score", "sirllm:decay_select", "sirllm:compact_kv", ...).
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     Calls validate their arguments on the host, enqueue work on that stream and
  *     return without synchronising (sirllm_status() is the exception).  Two calls
@@ -241,6 +244,19 @@ int sirllm_keep_policy(const sirllm_config *cfg, int32_t policy, const int32_t *
  * otherwise source and destination must not overlap.  Either of K or V may be NULL
  * (both src and dst) to skip it.  Every keep list must be strictly ascending within
  * [0, capacity) (else SIRLLM_STATUS_BAD_KEEP and the stream is left alone).
+ *
+ * What the gather needs from the device, and what a time-out leaves behind.  The kernel is a
+ * persistent grid (one CTA per SM, sized from the occupancy the runtime reports) whose workers
+ * draw units of work from a counter in `ws`; a plane may be cut into segments that different
+ * workers move, and a segment waits - a bounded number of polls - until the earlier segments of
+ * its plane have read the rows it is about to overwrite.  A worker only waits for units drawn
+ * before its own, by workers that are running, so the waits end however few CTAs the device
+ * keeps resident (a shared or partitioned GPU makes the call slower, not wrong).  If a wait
+ * does run out (a hung device, a workspace shared by two calls that overlap),
+ * SIRLLM_STATUS_TIMEOUT is raised, the worker stops storing and the kernel ends: an in-place
+ * cache is then PARTLY compacted - rows already stored are final, the others still hold what
+ * they held before - and the caller must treat the stream's cache as lost.  The same holds for
+ * sirllm_step and sirllm_step_pairs.
  */
 int sirllm_compact_kv(const sirllm_config *cfg, const void *k_src, const void *v_src, void *k_dst,
                       void *v_dst, const int32_t *keep_idx, const int32_t *n_keep, void *ws,

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 #include <stdint.h>
 
 #include "sirllm.h"
@@ -41,6 +42,15 @@ constexpr int kScoreCtaVecs = 4096;  // 16-byte vectors of one logits row per CT
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int logits_elem_bytes(int dtype) { return dtype == SIRLLM_F32 ? 4 : 2; }
+
+// A named NVTX range around the host side of a launch (tracing tools show it on the stream's
+// timeline; a handful of nanoseconds when no tool is attached).
+struct TraceRange {
+    explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+    ~TraceRange() { nvtxRangePop(); }
+    TraceRange(const TraceRange&) = delete;
+    TraceRange& operator=(const TraceRange&) = delete;
+};
 
 int validate_config(const sirllm_config* cfg);
 

@@ -522,11 +522,13 @@ cudaError_t launch_bounded_wait_selftest(unsigned long long* prog, const int32_t
 
 cudaError_t launch_compact_plan(const CompactParams& p, int n_streams, int32_t* first_moved,
                                 cudaStream_t st) {
+    TraceRange trace("sirllm:compact_plan");
     compact_plan_kernel<<<n_streams, 256, 0, st>>>(p, first_moved);
     return cudaGetLastError();
 }
 
 cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap) {
+    TraceRange trace("sirllm:compact_kv");
     int n_tensors = 0;
     CompactParams q = p;
     for (int t = 0; t < 2; ++t) {

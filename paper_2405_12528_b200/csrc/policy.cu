@@ -58,6 +58,7 @@ __global__ void policy_rank_kernel(const PolicyParams p) {
 }  // namespace
 
 cudaError_t launch_policy_ranks(const PolicyParams& p, int n_streams, cudaStream_t st) {
+    TraceRange trace("sirllm:keep_policy");
     dim3 grid((unsigned)((p.capacity + 255) / 256), (unsigned)n_streams);
     policy_rank_kernel<<<grid, 256, 0, st>>>(p);
     return cudaGetLastError();

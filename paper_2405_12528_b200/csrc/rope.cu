@@ -23,6 +23,10 @@ namespace sirllm {
 namespace {
 
 constexpr int kRopeThreads = 128;
+// six CTAs per SM (80 registers): measured best; eight spill the angles, five leave warps idle,
+// and four pairs per thread (half the angle registers) doubled the sincos work for no gain
+// (bf16; the fp16 conversions need more registers, so that variant is held to four CTAs)
+constexpr int kRopeMinBlocks = 6;
 
 // 16-bit element -> fp64, exactly (two conversions; bf16 -> fp32 is a shift).
 template <bool kBf16>
@@ -71,7 +75,7 @@ __device__ __forceinline__ void turn(double x, double y, double c, double s, dou
 }
 
 template <bool kBf16>
-__global__ void __launch_bounds__(kRopeThreads) rerotate_kernel(const RopeParams p) {
+__global__ void __launch_bounds__(kRopeThreads, kBf16 ? kRopeMinBlocks : 4) rerotate_kernel(const RopeParams p) {
     const int units = p.head_dim / 16;  // threads per row: 8 pairs (two 16-byte vectors) each
     const int rows_per_block = kRopeThreads / units;
     const int r = threadIdx.x / units, u = threadIdx.x - r * units;
@@ -151,6 +155,7 @@ __global__ void __launch_bounds__(kRopeThreads) rerotate_kernel(const RopeParams
 }  // namespace
 
 cudaError_t launch_rerotate(const RopeParams& p, int n_streams, bool bf16, cudaStream_t st) {
+    TraceRange trace("sirllm:rerotate_keys");
     const int units = p.head_dim / 16;
     const int rows_per_block = kRopeThreads / units;
     const unsigned gx = (unsigned)((p.keep_stride + rows_per_block - 1) / rows_per_block);

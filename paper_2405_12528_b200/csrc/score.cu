@@ -56,6 +56,46 @@ __device__ __forceinline__ uint32_t bf162_max(uint32_t a, uint32_t b) {
     return *reinterpret_cast<uint32_t*>(&m);
 }
 
+// One trip of a warp (kUnroll 16-byte vectors per lane) folded into the lane's running state.
+template <bool kBf16>
+__device__ __forceinline__ void reduce_trip(const uint4 (&x)[kUnroll], Online& st) {
+    if (kBf16) {
+        uint32_t m2 = x[0].x;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            m2 = bf162_max(m2, x[u].x);
+            m2 = bf162_max(m2, x[u].y);
+            m2 = bf162_max(m2, x[u].z);
+            m2 = bf162_max(m2, x[u].w);
+        }
+        st.raise(fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u)));
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const uint32_t w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                st.add0(__uint_as_float(w[q] << 16));
+                st.add1(__uint_as_float(w[q] & 0xFFFF0000u));
+            }
+        }
+    } else {
+        float gm = __uint_as_float(x[0].x);
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            gm = fmaxf(gm, fmaxf(fmaxf(__uint_as_float(x[u].x), __uint_as_float(x[u].y)),
+                                 fmaxf(__uint_as_float(x[u].z), __uint_as_float(x[u].w))));
+        }
+        st.raise(gm);
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            st.add0(__uint_as_float(x[u].x));
+            st.add1(__uint_as_float(x[u].y));
+            st.add0(__uint_as_float(x[u].z));
+            st.add1(__uint_as_float(x[u].w));
+        }
+    }
+}
+
 template <bool kBf16, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32)
 score_kernel(const ScoreParams p) {
@@ -76,16 +116,22 @@ score_kernel(const ScoreParams p) {
     int T = p.max_new;
     if (p.n_new != nullptr) T = min(p.n_new[s], p.max_new);
     if (t >= T) return;
-    // warp 0 finishes the row: fetch what it will need now, use it after the reduction
+    const int64_t V = p.vocab;
+    const char* rowp = (const char*)p.logits + row * p.row_stride * ES;
+    // warp 0 finishes the row: fetch what it will need now - the token id, the live length and
+    // the target logit itself - so that nothing is waited for after the reduction
     int32_t id = -1;
     int l0 = -1;
+    bool has_target = false;
+    float z_target = 0.f;
     if (wid == 0) {
         id = p.token_ids[row];
         if (p.scores != nullptr) l0 = p.live_len[s];
+        const int64_t col = (int64_t)id - (p.pairs_out != nullptr ? p.col0 : 0);
+        has_target = id >= 0 && col >= 0 && col < V;
+        if (has_target) z_target = load_logit(rowp, kBf16 ? SIRLLM_BF16 : SIRLLM_F32, col);
     }
 
-    const int64_t V = p.vocab;
-    const char* rowp = (const char*)p.logits + row * p.row_stride * ES;
     // elements in front of the first 16-byte boundary, whole vectors, elements after them
     int64_t head = (int64_t)(((16u - (uint32_t)((uintptr_t)rowp & 15u)) & 15u) / ES);
     if (head > V) head = V;
@@ -112,41 +158,7 @@ score_kernel(const ScoreParams p) {
     if (v0 < v1) fetch(v0, x);
     for (int64_t base = v0; base < v1; base += 32 * kUnroll) {
         fetch(base + 32 * kUnroll, xn);  // past the end: filled with -inf, never reduced
-        if (kBf16) {
-            uint32_t m2 = x[0].x;
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                m2 = bf162_max(m2, x[u].x);
-                m2 = bf162_max(m2, x[u].y);
-                m2 = bf162_max(m2, x[u].z);
-                m2 = bf162_max(m2, x[u].w);
-            }
-            st.raise(fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u)));
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                const uint32_t w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    st.add0(__uint_as_float(w[q] << 16));
-                    st.add1(__uint_as_float(w[q] & 0xFFFF0000u));
-                }
-            }
-        } else {
-            float gm = __uint_as_float(x[0].x);
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                gm = fmaxf(gm, fmaxf(fmaxf(__uint_as_float(x[u].x), __uint_as_float(x[u].y)),
-                                     fmaxf(__uint_as_float(x[u].z), __uint_as_float(x[u].w))));
-            }
-            st.raise(gm);
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                st.add0(__uint_as_float(x[u].x));
-                st.add1(__uint_as_float(x[u].y));
-                st.add0(__uint_as_float(x[u].z));
-                st.add1(__uint_as_float(x[u].w));
-            }
-        }
+        reduce_trip<kBf16>(x, st);
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) x[u] = xn[u];
     }
@@ -212,16 +224,12 @@ score_kernel(const ScoreParams p) {
             pr.y = (float)(acc * exp2((double)Mx - (double)pr.x * 1.4426950408889634));
         }
         p.pairs_out[row * p.pair_stride] = pr;
-        const int64_t col = (int64_t)id - p.col0;
-        p.target_out[row] = (id >= 0 && col >= 0 && col < V)
-                                ? load_logit(rowp, kBf16 ? SIRLLM_BF16 : SIRLLM_F32, col)
-                                : 0.f;
+        p.target_out[row] = has_target ? z_target : 0.f;
     } else if (lane == 0) {
         // e = ln(sum_v exp z_v) - z_id >= 0; id -1 = no prediction, other bad ids are flagged
         float e = 0.f;
-        if (id >= 0 && (int64_t)id < V) {
-            const float z = load_logit(rowp, kBf16 ? SIRLLM_BF16 : SIRLLM_F32, id);
-            e = fmaxf((float)(((double)Mx * kLn2 + log(acc)) - (double)z), 0.0f);
+        if (has_target) {
+            e = fmaxf((float)(((double)Mx * kLn2 + log(acc)) - (double)z_target), 0.0f);
         } else if (id != -1) {
             atomicOr(p.status, SIRLLM_STATUS_TOKEN_RANGE);
         }
@@ -280,6 +288,7 @@ __global__ void __launch_bounds__(128) score_pairs_kernel(const PairScoreParams 
 }  // namespace
 
 cudaError_t launch_score_pairs(const PairScoreParams& p, cudaStream_t st) {
+    TraceRange trace("sirllm:score_pairs");
     const int64_t rows = (int64_t)p.n_streams * p.max_new;
     if (rows == 0) return cudaSuccess;
     score_pairs_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(p);
@@ -290,6 +299,7 @@ cudaError_t launch_score_pairs(const PairScoreParams& p, cudaStream_t st) {
 // programmatic launch that let it become resident during the preceding gather was measured:
 // the parked CTAs slowed the gather by 2-3 %, and short rounds by more.)
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
+    TraceRange trace("sirllm:score");
     const int64_t ctas = (int64_t)p.n_streams * p.max_new * p.n_part;
     if (ctas == 0) return cudaSuccess;
     if (ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;
@@ -300,9 +310,9 @@ cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
     DeviceProps dp;
     cudaError_t e = device_props(&dp);
     if (e != cudaSuccess) return e;
+    const bool bf16 = p.logits_dtype == SIRLLM_BF16;
     const int64_t want_warps = (int64_t)dp.n_sm * 8;
     const int warps = ctas * 4 >= want_warps ? 4 : (ctas * 8 >= want_warps ? 8 : 16);
-    const bool bf16 = p.logits_dtype == SIRLLM_BF16;
     if (warps == 4) {
         if (bf16) score_kernel<true, 4><<<grid, 128, 0, st>>>(p);
         else score_kernel<false, 4><<<grid, 128, 0, st>>>(p);

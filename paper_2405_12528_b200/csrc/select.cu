@@ -382,6 +382,7 @@ __global__ void __launch_bounds__(kSelectThreads, 1) select_kernel(const SelectP
 }  // namespace
 
 cudaError_t launch_select(const SelectParams& p, int n_streams, cudaStream_t st, bool overlap) {
+    TraceRange trace("sirllm:decay_select");
     // scores (rounded up to whole 128-bit vectors, plus one vector of slack) + histogram
     // (+ the staged keep list when it fits)
     size_t smem = ((size_t)((p.capacity + 3) & ~3) + 4) * 4 + (size_t)kRadixBins * 4;
