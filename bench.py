@@ -50,7 +50,7 @@ FALLBACK_HBM_GBS = 6650.0
 # while the kernel's source file is the one the counters were taken on.
 NCU_CAPTURE = {"kernel": "compact_kernel", "workload": "mistral_7b_gqa",
                "dram_bytes": 536657920 + 482415872, "algorithmic_bytes": 2 * 4092 * 256 * 512,
-               "sources": {"paper_2405_12528_b200/csrc/compact.cu": "b71de8e9c9d43530705046707caf9b5d1031c6fe"}}
+               "sources": {"paper_2405_12528_b200/csrc/compact.cu": "fd1fad75a4a9bf202015cb8d41ed844036efac39"}}
 
 
 def ncu_traffic(bytes_per_launch):

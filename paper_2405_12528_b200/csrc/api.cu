@@ -172,7 +172,7 @@ int sirllm_score(const sirllm_config* cfg, const void* logits, const int32_t* to
     const WorkspaceLayout L = workspace_layout(*cfg);
     ScoreParams sp = score_params(*cfg, L, logits, token_ids, n_new, ws);
     sp.out_entropy = out_entropy;
-    cudaError_t e = launch_score(sp, (cudaStream_t)cuda_stream);
+    cudaError_t e = launch_score(sp, (cudaStream_t)cuda_stream, false);
     return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "score");
 }
 
@@ -200,7 +200,7 @@ int sirllm_score_partial(const sirllm_config* cfg, const void* logits_slice, int
     range.vocab = n_cols > 0 ? n_cols : 1;
     range.logits_row_stride = range.vocab;
     sp.n_part = workspace_layout(range).n_part;
-    cudaError_t e = launch_score(sp, (cudaStream_t)cuda_stream);
+    cudaError_t e = launch_score(sp, (cudaStream_t)cuda_stream, false);
     return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "score_partial");
 }
 
@@ -371,6 +371,7 @@ struct StepPlan {
     SelectParams sp;
     CompactParams cp;
     int n_streams;
+    bool small_gather;  // the round's gather is the small two-phase kernel
 };
 
 // Host-side validation of a whole round; touches no device and enqueues nothing.
@@ -404,7 +405,10 @@ static int step_prepare(const sirllm_config* cfg, const ScoreSource& src, const 
     plan->sp.max_new = cfg->max_new;
     plan->sp.compact_scores = 1;
     plan->sp.score_new = 1;
-    return compact_params(*cfg, L, k, v, k, v, plan->sp.keep_idx, plan->sp.n_keep, ws, &plan->cp);
+    rc = compact_params(*cfg, L, k, v, k, v, plan->sp.keep_idx, plan->sp.n_keep, ws, &plan->cp);
+    const int64_t planes = ((k != nullptr) + (v != nullptr)) * plan->cp.planes_per_tensor;
+    plan->small_gather = planes > 0 && compact_is_small_job(planes, plan->cp.keep_stride, plan->cp.row_bytes);
+    return rc;
 }
 
 // The round's three launches (with `ev`: four event records around them, and no overlap
@@ -415,7 +419,9 @@ static int step_enqueue(const StepPlan& plan, cudaStream_t st, void** ev) {
     if (ev && (e = cudaEventRecord((cudaEvent_t)ev[i], st)) != cudaSuccess) \
         return cuda_fail(e, "cudaEventRecord");
     SIRLLM_MARK(0)
-    e = plan.from_pairs ? launch_score_pairs(plan.pp, st) : launch_score(plan.sc, st);
+    // the scorer may overlap the end of a preceding small gather (see launch_score)
+    const bool early = ev == nullptr && plan.small_gather;
+    e = plan.from_pairs ? launch_score_pairs(plan.pp, st, early) : launch_score(plan.sc, st, early);
     if (e != cudaSuccess) return cuda_fail(e, "score");
     SIRLLM_MARK(1)
     // the selection kernel reads the caller's buffers before it waits for its predecessor: it may
@@ -468,7 +474,7 @@ int sirllm_score_pairs(const sirllm_config* cfg, const void* pairs, int32_t n_ti
     if ((rc = check_pairs(src)) != SIRLLM_OK) return rc;
     PairScoreParams pp = pair_params(*cfg, src, token_ids, n_new, ws);
     pp.out_entropy = out_entropy;
-    cudaError_t e = launch_score_pairs(pp, (cudaStream_t)cuda_stream);
+    cudaError_t e = launch_score_pairs(pp, (cudaStream_t)cuda_stream, false);
     return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "score_pairs");
 }
 

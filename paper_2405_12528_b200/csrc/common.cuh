@@ -156,8 +156,13 @@ struct CompactParams {
     int32_t in_place;
 };
 
-cudaError_t launch_score(const ScoreParams& p, cudaStream_t st);
-cudaError_t launch_score_pairs(const PairScoreParams& p, cudaStream_t st);
+// `overlap`: launch with programmatic stream serialization (the kernels wait for their
+// predecessor themselves), so that the grid may become resident while a predecessor that
+// releases its dependents early is ending.
+cudaError_t launch_score(const ScoreParams& p, cudaStream_t st, bool overlap);
+cudaError_t launch_score_pairs(const PairScoreParams& p, cudaStream_t st, bool overlap);
+// true if a gather over `planes` K and V planes goes to the small two-phase kernel
+bool compact_is_small_job(int64_t planes, int keep_stride, int row_bytes);
 // `overlap`: launch with programmatic stream serialization, so the grid may become resident
 // while the previous kernel on the stream drains; the kernel itself waits for that kernel's
 // results (grid_dependency_wait) before it reads them.

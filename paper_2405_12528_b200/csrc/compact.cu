@@ -450,6 +450,9 @@ compact_small_kernel(const CompactParams p, const int col_splits) {
                 dst[(size_t)(f + i / slice_vecs) * row_vecs + i % slice_vecs] = staged[i];
         }
     }
+    // a kernel launched programmatically behind this grid (the next round's scorer) may become
+    // resident from here on; it waits for the whole grid itself before it reads anything
+    grid_launch_dependents();
     // not complete before the grid this one depends on is (see compact_kernel)
     if (threadIdx.x == 0) grid_dependency_wait();
 }
@@ -527,6 +530,10 @@ cudaError_t launch_compact_plan(const CompactParams& p, int n_streams, int32_t* 
     return cudaGetLastError();
 }
 
+bool compact_is_small_job(int64_t planes, int keep_stride, int row_bytes) {
+    return planes * keep_stride * row_bytes <= kSmallJobBytes;
+}
+
 cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap) {
     TraceRange trace("sirllm:compact_kv");
     int n_tensors = 0;
@@ -557,7 +564,7 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     // plane and column slice (slices of at least 32 bytes, as many as it takes to occupy the
     // SMs), provided a slice of the longest keep list fits in shared memory
     const int row_vecs = p.row_bytes / 16;
-    if ((int64_t)units_base * p.keep_stride * p.row_bytes <= kSmallJobBytes) {
+    if (compact_is_small_job(units_base, p.keep_stride, p.row_bytes)) {
         int col_splits = 1;
         while (col_splits * 2 <= row_vecs / 2 && row_vecs % (col_splits * 2) == 0 &&
                (int64_t)units_base * col_splits < 2 * n_sm)

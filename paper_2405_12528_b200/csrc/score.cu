@@ -104,8 +104,11 @@ score_kernel(const ScoreParams p) {
     constexpr int EPV = 16 / ES;
     __shared__ float2 warp_pair[kWarps];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    // the selection kernel may become resident while this grid drains (it waits for this grid's
-    // scores itself); this grid starts only after everything before it on the stream is complete
+    // Possibly launched with programmatic serialization: behind a kernel that lets its dependents
+    // go early (the small gather does, at its end) this grid becomes resident while that kernel
+    // ends, which hides the launch latency; nothing is read before that kernel has completed.  Only then may the kernel that follows (the selection) start to become
+    // resident: what it reads ahead of its own wait is then settled as well.
+    grid_dependency_wait();
     grid_launch_dependents();
     // one CTA = kWarps consecutive segments of one logits row
     const int64_t row = blockIdx.x / p.n_part;
@@ -247,6 +250,7 @@ score_kernel(const ScoreParams p) {
 __global__ void __launch_bounds__(128) score_pairs_kernel(const PairScoreParams p) {
     const int lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    grid_dependency_wait();
     grid_launch_dependents();
     if (row >= (int64_t)p.n_streams * p.max_new) return;
     const int s = (int)(row / p.max_new);
@@ -287,18 +291,37 @@ __global__ void __launch_bounds__(128) score_pairs_kernel(const PairScoreParams 
 
 }  // namespace
 
-cudaError_t launch_score_pairs(const PairScoreParams& p, cudaStream_t st) {
+// A launch that may become resident before the preceding kernel on the stream has finished
+// (programmatic stream serialization); the kernels wait for that kernel themselves.
+template <typename Kernel, typename Params>
+static cudaError_t launch_overlapped(Kernel kernel, unsigned grid, unsigned block, cudaStream_t st,
+                                     const Params& p, bool overlap) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
+cudaError_t launch_score_pairs(const PairScoreParams& p, cudaStream_t st, bool overlap) {
     TraceRange trace("sirllm:score_pairs");
     const int64_t rows = (int64_t)p.n_streams * p.max_new;
     if (rows == 0) return cudaSuccess;
-    score_pairs_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(p);
-    return cudaGetLastError();
+    return launch_overlapped(score_pairs_kernel, (unsigned)((rows + 3) / 4), 128, st, p, overlap);
 }
 
-// Launched plainly: the grid starts once everything before it on the stream is complete.  (A
-// programmatic launch that let it become resident during the preceding gather was measured:
-// the parked CTAs slowed the gather by 2-3 %, and short rounds by more.)
-cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
+// With `overlap` the launch is programmatic (see the kernel).  The fused round asks for it only
+// where the round's gather is the small two-phase kernel, which releases its dependents at its
+// end: tiny rounds gain 1.5 us of launch latency.  Behind the persistent gather it was measured
+// and rejected: released early, the parked scorer CTAs slowed the gather by 2-3 %; released at
+// the gather's end, the scorer ran slower on SMs still set up for the gather's shared memory.
+cudaError_t launch_score(const ScoreParams& p, cudaStream_t st, bool overlap) {
     TraceRange trace("sirllm:score");
     const int64_t ctas = (int64_t)p.n_streams * p.max_new * p.n_part;
     if (ctas == 0) return cudaSuccess;
@@ -318,17 +341,14 @@ cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
     // three waves of CTAs half as long (measured -2 us on 2048 rows of 32000 bf16 logits).
     const int64_t one_wave = (int64_t)dp.n_sm * 10;
     if (warps == 4 && ctas > one_wave && ctas <= 2 * one_wave) warps = 8;
-    if (warps == 4) {
-        if (bf16) score_kernel<true, 4><<<grid, 128, 0, st>>>(p);
-        else score_kernel<false, 4><<<grid, 128, 0, st>>>(p);
-    } else if (warps == 8) {
-        if (bf16) score_kernel<true, 8><<<grid, 256, 0, st>>>(p);
-        else score_kernel<false, 8><<<grid, 256, 0, st>>>(p);
-    } else {
-        if (bf16) score_kernel<true, 16><<<grid, 512, 0, st>>>(p);
-        else score_kernel<false, 16><<<grid, 512, 0, st>>>(p);
-    }
-    return cudaGetLastError();
+    if (warps == 4)
+        return bf16 ? launch_overlapped(score_kernel<true, 4>, grid, 128, st, p, overlap)
+                    : launch_overlapped(score_kernel<false, 4>, grid, 128, st, p, overlap);
+    if (warps == 8)
+        return bf16 ? launch_overlapped(score_kernel<true, 8>, grid, 256, st, p, overlap)
+                    : launch_overlapped(score_kernel<false, 8>, grid, 256, st, p, overlap);
+    return bf16 ? launch_overlapped(score_kernel<true, 16>, grid, 512, st, p, overlap)
+                : launch_overlapped(score_kernel<false, 16>, grid, 512, st, p, overlap);
 }
 
 }  // namespace sirllm
@@ -419,6 +439,6 @@ extern "C" int sirllm_score_static(const sirllm_config* cfg, const void* logits,
     sp.n_part = L.n_part;
     sp.logits_dtype = cfg->logits_dtype;
     sp.capacity = cfg->capacity;
-    e = launch_score(sp, st);
+    e = launch_score(sp, st, false);
     return e == cudaSuccess ? SIRLLM_OK : cuda_fail(e, "score");
 }
