@@ -325,6 +325,66 @@ def test_step_paper_cache_shapes_and_decay_ratios(name, eta):
     assert st.host_len == [w.budget]
 
 
+def _random_shape(seed: int):
+    """A seeded random configuration: every size that a kernel tiles over is drawn, so that row
+    widths, vocabulary tails, window splits and stream counts off the measured shapes are met."""
+    import random
+    g = random.Random(1000 + seed)
+    head_dim = g.choice([8, 16, 40, 64, 80, 96, 128, 160, 256])
+    n_streams = g.choice([1, 1, 2, 3, 5])
+    wide = seed % 2 == 1          # enough planes and rows for the persistent (ring) gather
+    budget = g.randrange(300, 700) if wide else g.randrange(8, 700)
+    n_sink = g.randrange(0, min(9, budget + 1))
+    n_recent = g.randrange(0, budget - n_sink + 1) if g.random() < 0.7 else 0
+    if g.random() < 0.15:
+        n_recent = budget - n_sink                       # k = 0: nothing chosen by score
+    new_tokens = g.randrange(1, 2 * budget) if g.random() < 0.8 else g.randrange(1, 40)
+    capacity = budget + new_tokens + g.randrange(0, 64)
+    vocab = g.choice([g.randrange(2, 300), g.randrange(300, 9000), g.randrange(9000, 70000)])
+    return wl.WORKLOADS["tiny"].scaled(
+        name=f"random{seed}", n_streams=n_streams,
+        n_layers=g.randrange(6, 13) if wide else g.randrange(1, 4),
+        n_kv_heads=g.randrange(4, 9) if wide else g.randrange(1, 5), head_dim=head_dim, capacity=capacity, budget=budget,
+        n_sink=n_sink, n_recent=n_recent, new_tokens=new_tokens, vocab=vocab,
+        logits_dtype=g.choice(["f32", "bf16"]), kv_dtype=g.choice(["f16", "bf16"]),
+        decay=g.choice([0.5, 0.7, 0.9, 1.0]), decay_hi=None)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_step_random_configurations(seed):
+    # whole rounds on drawn shapes (ragged lengths on the multi-stream ones): scores, keep lists,
+    # compacted scores, tags and K/V against the oracle every round
+    w = _random_shape(seed)
+    rounds = max(4, min(12, 3 * w.budget // max(1, w.new_tokens) + 3))
+    _run_stream(w, rounds, ragged=w.n_streams > 1, seed=seed)
+
+
+def test_retained_tokens_overlap_with_a_run_on_the_oracles_own_scores():
+    # Every other whole-round test hands the oracle the GPU's scores, so that index sets can be
+    # compared bit for bit.  Here the oracle runs alone, on its OWN fp64-derived scores, and
+    # the retained TOKENS (serial tags) are compared as sets: scores that differ in the last
+    # fp32 digits may swap two near-equal candidates at the cut, nothing more.  The overlap
+    # (intersection over union) is printed and must stay above 0.99 in every round.
+    w = wl.WORKLOADS["mistral_7b_gqa"].scaled(n_layers=1, n_kv_heads=1, capacity=1536, budget=1024,
+                                              n_recent=128, new_tokens=256, vocab=5003)
+    st = DeviceState(w)
+    tw = oracle_twin(w, st.decay.cpu(), with_kv=False)[0]
+    worst = 1.0
+    for r in range(16):
+        st.fill_round(r)
+        T = w.new_tokens
+        st.step()
+        assert B.sirllm_status(st.ws) == 0
+        tw.step(oracle.score(st.logits[:T].cpu(), st.token_ids[:T].cpu()))
+        n = tw.live_len
+        assert st.host_len[0] == n
+        got = set(st.serial[0, :n].cpu().tolist())
+        want = set(tw.serial[:n].tolist())
+        worst = min(worst, len(got & want) / len(got | want))
+    print(f"retained-token overlap with the pure-oracle run, worst round: {worst:.5f}")
+    assert worst > 0.99
+
+
 def test_step_host_refused_call_leaves_the_device_untouched():
     # a bad value for the SECOND stream: nothing of the first stream may have been copied
     w = wl.WORKLOADS["batched64"].scaled(n_streams=2, n_layers=1, n_kv_heads=2, capacity=256,
