@@ -104,9 +104,10 @@ score_kernel(const ScoreParams p) {
     constexpr int EPV = 16 / ES;
     __shared__ float2 warp_pair[kWarps];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    // Possibly launched with programmatic serialization: behind a kernel that lets its dependents
-    // go early (the small gather does, at its end) this grid becomes resident while that kernel
-    // ends, which hides the launch latency; nothing is read before that kernel has completed.  Only then may the kernel that follows (the selection) start to become
+    // Possibly launched with programmatic serialization: behind a kernel that lets its
+    // dependents go early (the small gather does, at its end) this grid becomes resident while
+    // that kernel ends, which hides the launch latency; nothing is read before that kernel has
+    // completed.  Only then may the kernel that follows (the selection) start to become
     // resident: what it reads ahead of its own wait is then settled as well.
     grid_dependency_wait();
     grid_launch_dependents();

@@ -64,10 +64,13 @@ class DeviceState:
         self.n_new.copy_(torch.tensor(n_new, dtype=torch.int32))
         return n_new
 
-    def step(self):
+    def enqueue_step(self):
         B.sirllm_step(self.cfg, self.logits, self.token_ids, self.n_new, self.scores, self.serial,
                       self.live_len, self.decay, self.k, self.v, self.keep_idx, self.n_keep,
                       self.new_entropy, self.ws)
+
+    def step(self):
+        self.enqueue_step()
         self.host_len = self.live_len.cpu().tolist()
 
     def check_kv_by_content(self, streams=None):

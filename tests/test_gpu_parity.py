@@ -250,8 +250,9 @@ def test_compact_identity_list_moves_nothing_and_bad_lists_are_refused():
 
 # ------------------------------------------------------------------------------- whole rounds
 
-def _run_stream(w, rounds, ragged=False, seed=0, check_kv_host=True, rho=None):
+def _run_stream(w, rounds, ragged=False, seed=0, check_kv_host=True, rho=None, via_graph=False):
     st = DeviceState(w, seed=seed)
+    graph = None
     twins = oracle_twin(w, st.decay.cpu())
     M = st.cfg.max_new
     for r in range(rounds):
@@ -263,7 +264,18 @@ def _run_stream(w, rounds, ragged=False, seed=0, check_kv_host=True, rho=None):
         e_gpu = torch.zeros_like(st.new_entropy)
         B.sirllm_score(st.cfg, st.logits, st.token_ids, st.n_new, e_gpu, st.ws)
         before = [t.live_len for t in twins]
-        st.step()
+        if via_graph and r > 0:
+            if graph is None:   # the first round ran eagerly; every later one is a replay
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    st.enqueue_step()
+                torch.cuda.current_stream().wait_stream(side)
+            graph.replay()
+            st.host_len = st.live_len.cpu().tolist()
+        else:
+            st.step()
         assert B.sirllm_status(st.ws) == 0
         e_gpu = e_gpu.cpu()
         for s, tw in enumerate(twins):
@@ -323,6 +335,18 @@ def test_step_paper_cache_shapes_and_decay_ratios(name, eta):
     rounds = 24 if name == "dailydialog_512" else 40
     st = _run_stream(w, rounds)
     assert st.host_len == [w.budget]
+
+
+def test_step_replayed_from_a_cuda_graph():
+    # the round is three kernel launches chained by programmatic dependent launch and touches
+    # no host state, so it can be captured once and replayed: every replayed round against the
+    # oracle (ragged lengths arrive through device memory, not through the captured arguments)
+    w = wl.WORKLOADS["batched64"].scaled(n_streams=3, n_layers=2, n_kv_heads=2, capacity=512,
+                                         budget=256, n_recent=64, new_tokens=100, vocab=4099)
+    _run_stream(w, 8, ragged=True, via_graph=True)
+    w = wl.WORKLOADS["mistral_7b_gqa"].scaled(n_layers=8, n_kv_heads=8, capacity=1536, budget=1024,
+                                              n_recent=128, new_tokens=200, vocab=5003)
+    _run_stream(w, 8, via_graph=True)      # wide enough for the persistent gather
 
 
 def _random_shape(seed: int):
