@@ -231,6 +231,15 @@ def test_compact_matches_gather(in_place):
     _compact_case(2, 3, 200, 512, [150, 199], in_place, 5)                 # 1 KB rows: the largest
 
 
+@pytest.mark.parametrize("in_place", [True, False])
+def test_compact_row_widths_through_the_persistent_gather(in_place):
+    # jobs of tens of MB (the ring kernel, not the two-phase one) at the narrowest row, an odd
+    # multiple of 16 bytes, and the widest row (one worker per CTA)
+    _compact_case(4, 512, 600, 8, [500, 600, 1, 77], in_place, 6)           # 16-byte rows
+    _compact_case(2, 256, 500, 40, [400, 123], in_place, 7, torch.float16)  # 80-byte rows
+    _compact_case(1, 64, 300, 512, [250], in_place, 8)                      # 1 KB rows
+
+
 def test_compact_identity_list_moves_nothing_and_bad_lists_are_refused():
     cfg = B.make_config(2, 2, 1, 16, 40, 20, 0, 0, 0, 16, torch.float32, torch.bfloat16)
     ws = B.new_workspace(cfg)
