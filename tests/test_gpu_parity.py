@@ -870,6 +870,66 @@ def test_rerotate_keys_matches_oracle(dtype, layout):
     assert n_off <= 1e-3 * n_elems, (n_off, n_elems)
 
 
+def _rerotate_case(S, P, cap, D, thr, n_list, fixed, dtype, layout, seed, scale=2.0, exponent_spread=0):
+    """Random keys, keep lists whose first `fixed` rows stay put; every plane against the oracle."""
+    cfg = B.make_config(S, P, 1, D, cap, thr, 0, 0, 0, 16, torch.float32, dtype)
+    g = torch.Generator().manual_seed(seed)
+    k = torch.randn(S, P, cap, D, generator=g) * scale
+    if exponent_spread:                  # magnitudes spread over many binades, down into the subnormals
+        k = k * torch.exp2(-torch.randint(0, exponent_spread, k.shape, generator=g).float())
+    k = k.to(dtype)
+    keep = torch.full((S, thr), -1, dtype=torch.int32)
+    for s, n in enumerate(n_list):
+        f = min(fixed, n)
+        picked = torch.sort(torch.randperm(cap - f, generator=g)[:n - f]).values + f
+        keep[s, :n] = torch.cat([torch.arange(f), picked]).to(torch.int32)
+    dk = k.to(DEV)
+    B.sirllm_rerotate_keys(cfg, dk, keep.to(DEV), torch.tensor(n_list, dtype=torch.int32, device=DEV),
+                           10000.0, layout)
+    got = dk.cpu()
+    n_elems = n_off = 0
+    for s, n in enumerate(n_list):
+        for p in range(P):
+            want = oracle.rerotate_plane(k[s, p], keep[s, :n], 10000.0, layout)
+            assert torch.equal(got[s, p, n:], k[s, p, n:])                     # beyond the live rows
+            d = (_ordered16(got[s, p, :n]) - _ordered16(want[:n])).abs()
+            assert int(d.max()) <= 1 if n else True
+            n_off += int((d != 0).sum())
+            n_elems += d.numel()
+    assert n_off <= 1e-3 * max(n_elems, 1), (n_off, n_elems)
+    return n_off, n_elems
+
+
+@pytest.mark.parametrize("layout", [B.ROPE_HALF, B.ROPE_INTERLEAVED])
+def test_rerotate_work_split_over_streams_row_groups_and_planes(layout):
+    # the kernel cuts (stream, row group, plane) lists into equal shares per block: many short
+    # streams, streams that moved nothing or are empty, one long stream with few planes, plane
+    # counts that no share divides, row widths with 5, 16 and 32 threads per row
+    _rerotate_case(9, 5, 90, 64, 64, [64, 0, 17, 64, 1, 33, 64, 2, 50], 3, torch.bfloat16, layout, 31)
+    _rerotate_case(3, 7, 300, 80, 200, [200, 199, 200], 200, torch.float16, layout, 32)   # nothing moved
+    _rerotate_case(1, 1, 9000, 128, 6000, [6000], 2500, torch.bfloat16, layout, 33)
+    _rerotate_case(2, 13, 400, 256, 256, [256, 101], 0, torch.float16, layout, 34)
+    _rerotate_case(1, 3, 200, 512, 128, [77], 5, torch.bfloat16, layout, 35)
+    _rerotate_case(40, 2, 64, 16, 48, [48 - (s % 5) for s in range(40)], 1, torch.bfloat16, layout, 36)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+def test_rerotate_rounds_tiny_and_subnormal_results_once(dtype):
+    # keys spread over 60 binades, ending below the smallest normal number of the type (and, for
+    # bf16, of fp32): results that are subnormal, that cancel to almost nothing or round to zero
+    # must still be the fp64 rotation rounded once
+    scale = 2.0 ** -100 if dtype == torch.bfloat16 else 2.0 ** -4
+    exact_zero = _rerotate_case(2, 3, 500, 128, 300, [300, 210], 4, dtype, B.ROPE_HALF, 41, scale, 40)
+    assert exact_zero[1] > 0
+    _rerotate_case(1, 2, 260, 64, 200, [200], 0, dtype, B.ROPE_INTERLEAVED, 42, scale, 40)
+    # rows of zeros (padding) stay zeros
+    cfg = B.make_config(1, 2, 1, 64, 100, 50, 0, 0, 0, 16, torch.float32, dtype)
+    z = torch.zeros(1, 2, 100, 64, dtype=dtype, device=DEV)
+    keep = (torch.arange(50, dtype=torch.int32) * 2).view(1, 50).to(DEV)
+    B.sirllm_rerotate_keys(cfg, z, keep, torch.tensor([50], dtype=torch.int32, device=DEV), 10000.0, B.ROPE_HALF)
+    assert int(z.view(torch.int16).abs().max()) == 0
+
+
 def test_rerotate_after_compaction_equals_keys_written_at_their_new_positions():
     # keys are stored rotated for the slot they were written to; after eviction + re-indexing
     # every kept key must equal (to storage rounding) the same token's key rotated for its new slot
