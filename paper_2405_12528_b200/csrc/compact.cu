@@ -50,7 +50,7 @@ constexpr int kIdxAhead = 4;     // chunks whose source indices are fetched ahea
 constexpr int kMaxWorkers = 4;   // worker warps per CTA
 constexpr int kPublishEvery = 4; // chunks between two updates of a segment's progress word
 constexpr int kNoBound = 0x7FFFFFFF;
-constexpr int kUnitsPerWorker = 34;  // work units per worker the split of the planes aims at
+constexpr int kUnitsPerWorker = 16;  // work units per worker the split of the planes aims at
 constexpr int kMinSegChunks = 5;     // shortest segment (chunks) worth a unit's set-up
 constexpr int64_t kSmallJobBytes = 8 << 20;  // planes x longest keep list x row: the two-phase kernel's range
 
@@ -616,14 +616,16 @@ cudaError_t launch_compact(const CompactParams& p, cudaStream_t st, bool overlap
     }
     if (per_sm < 1) return cudaErrorLaunchOutOfResources;
     const int64_t resident = (int64_t)n_sm * per_sm;
-    // Cut planes into segments so that every worker draws a few dozen units: the ticket
+    // Cut planes into segments so that every worker draws a dozen or two units: the ticket
     // hand-out then evens out SMs of different speed down to a small tail, while a unit stays
     // long enough to amortise its set-up.  Segments are a fixed number of chunks long
     // (`seg_chunks`), chosen ODD: planes are a power of two apart, so segments of 2^k chunks
     // would make all workers walk addresses that differ by large powers of two at the same
-    // time, which measured 2-3 % slower than odd lengths around the same size.  Around 34 units
-    // per worker measured best over the shapes tried (20 to 40 are within a percent; 14 and 55
-    // are worse).
+    // time, which measured 2-3 % slower than odd lengths around the same size.  About 16 units
+    // per worker measured best over the shapes tried: with 2048 planes of 64 chunks (planes 1 MB
+    // apart) segments of 15 to 21 chunks are 4-5 % faster than segments of 7; elsewhere 10 to 30
+    // units per worker are within a percent, below 7 the tail shows.  The last, shorter segment
+    // of every plane is handed out last and keeps that tail fine.
     const int64_t slots = resident * workers;
     const int64_t chunks_max = (p.keep_stride + kChunkRows - 1) / kChunkRows;
     int64_t seg_chunks = chunks_max;  // one segment per plane
