@@ -49,8 +49,8 @@ FALLBACK_HBM_GBS = 6650.0
 # in proportion to the moved bytes, so it is scaled to the timed launch; it is reported only
 # while the kernel's source file is the one the counters were taken on.
 NCU_CAPTURE = {"kernel": "compact_kernel", "workload": "mistral_7b_gqa",
-               "dram_bytes": 536657920 + 482415872, "algorithmic_bytes": 2 * 4092 * 256 * 512,
-               "sources": {"paper_2405_12528_b200/csrc/compact.cu": "fd1fad75a4a9bf202015cb8d41ed844036efac39"}}
+               "dram_bytes": 536590592 + 483479808, "algorithmic_bytes": 2 * 4092 * 256 * 512,
+               "sources": {"paper_2405_12528_b200/csrc/compact.cu": "5d3d22e8a1dc3b3c1bbd622d7cdec1b133a12df8"}}
 
 
 def ncu_traffic(bytes_per_launch):

@@ -870,7 +870,8 @@ def test_rerotate_keys_matches_oracle(dtype, layout):
     assert n_off <= 1e-3 * n_elems, (n_off, n_elems)
 
 
-def _rerotate_case(S, P, cap, D, thr, n_list, fixed, dtype, layout, seed, scale=2.0, exponent_spread=0):
+def _rerotate_case(S, P, cap, D, thr, n_list, fixed, dtype, layout, seed, scale=2.0, exponent_spread=0,
+                   base=10000.0):
     """Random keys, keep lists whose first `fixed` rows stay put; every plane against the oracle."""
     cfg = B.make_config(S, P, 1, D, cap, thr, 0, 0, 0, 16, torch.float32, dtype)
     g = torch.Generator().manual_seed(seed)
@@ -885,12 +886,12 @@ def _rerotate_case(S, P, cap, D, thr, n_list, fixed, dtype, layout, seed, scale=
         keep[s, :n] = torch.cat([torch.arange(f), picked]).to(torch.int32)
     dk = k.to(DEV)
     B.sirllm_rerotate_keys(cfg, dk, keep.to(DEV), torch.tensor(n_list, dtype=torch.int32, device=DEV),
-                           10000.0, layout)
+                           base, layout)
     got = dk.cpu()
     n_elems = n_off = 0
     for s, n in enumerate(n_list):
         for p in range(P):
-            want = oracle.rerotate_plane(k[s, p], keep[s, :n], 10000.0, layout)
+            want = oracle.rerotate_plane(k[s, p], keep[s, :n], base, layout)
             assert torch.equal(got[s, p, n:], k[s, p, n:])                     # beyond the live rows
             d = (_ordered16(got[s, p, :n]) - _ordered16(want[:n])).abs()
             assert int(d.max()) <= 1 if n else True
@@ -911,6 +912,9 @@ def test_rerotate_work_split_over_streams_row_groups_and_planes(layout):
     _rerotate_case(2, 13, 400, 256, 256, [256, 101], 0, torch.float16, layout, 34)
     _rerotate_case(1, 3, 200, 512, 128, [77], 5, torch.bfloat16, layout, 35)
     _rerotate_case(40, 2, 64, 16, 48, [48 - (s % 5) for s in range(40)], 1, torch.bfloat16, layout, 36)
+    # shifts of tens of thousands of positions (the largest cache the library takes) at a large base
+    _rerotate_case(1, 2, 49152, 128, 600, [600], 0, torch.bfloat16, layout, 37, base=500000.0)
+    _rerotate_case(1, 1, 49152, 64, 300, [300], 0, torch.float16, layout, 38, base=1.0e6)
 
 
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
