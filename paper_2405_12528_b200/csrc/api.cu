@@ -601,7 +601,8 @@ int sirllm_rerotate_keys(const sirllm_config* cfg, void* k, const int32_t* keep_
     p.k = (char*)k;
     p.keep_idx = keep_idx;
     p.n_keep = n_keep;
-    p.log2_base = std::log2(rope_base);
+    for (int i = 0; i < cfg->head_dim / 2; ++i)
+        p.theta[i] = std::pow(rope_base, -2.0 * (double)i / (double)cfg->head_dim);
     p.capacity = cfg->capacity;
     p.keep_stride = cfg->threshold;
     p.planes_per_stream = cfg->n_layers * cfg->n_kv_heads;

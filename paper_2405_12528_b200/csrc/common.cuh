@@ -135,7 +135,8 @@ struct RopeParams {
     char* k;
     const int32_t* keep_idx;
     const int32_t* n_keep;
-    double log2_base;
+    // theta_i = base^(-2i/d) for the d/2 pairs of a row, computed once per call on the host (pow)
+    double theta[SIRLLM_MAX_HEAD_DIM / 2];
     int32_t capacity, keep_stride, planes_per_stream, head_dim, layout, planes_per_group;
 };
 

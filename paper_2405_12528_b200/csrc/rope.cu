@@ -15,6 +15,8 @@
 // planes are in flight while one plane is turned.  What limits the kernel is not DRAM but the
 // four conversions between fp32 and fp64 per pair: they run on the quarter-rate conversion
 // pipe, which the counters show as the busiest unit (about 0.8 of the copy bandwidth is reached).
+#include <atomic>
+
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -29,6 +31,7 @@ constexpr int kRopeThreads = 128;
 // and four pairs per thread (half the angle registers) doubled the sincos work for no gain
 // (bf16; the fp16 conversions need more registers, so that variant is held to four CTAs)
 constexpr int kRopeMinBlocks = 6;
+constexpr int kRopeWaves = 3;  // grid size in resident waves
 
 // 16-bit element -> fp64, exactly (two conversions; bf16 -> fp32 is a shift).
 template <bool kBf16>
@@ -142,9 +145,8 @@ __global__ void __launch_bounds__(kRopeThreads, kBf16 ? kRopeMinBlocks : 4) rero
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
         const int i = 8 * u + q;
-        const double theta = exp2(-(double)(2 * i) / (double)p.head_dim * p.log2_base);
         double sv, cv;
-        sincos((double)delta * theta, &sv, &cv);
+        sincos((double)delta * p.theta[i], &sv, &cv);
         cs[q] = cv;
         sn[q] = sv;
     }
@@ -200,11 +202,24 @@ cudaError_t launch_rerotate(const RopeParams& p, int n_streams, bool bf16, cudaS
     DeviceProps dp;
     cudaError_t e = device_props(&dp);
     if (e != cudaSuccess) return e;
-    const int n_sm = dp.n_sm;
-    // about 16 blocks per SM, i.e. a few waves of the six resident ones: each block reuses its
-    // angles over a group of planes, and later waves even out SMs of different speed (measured:
-    // 8 per SM 7 % slower, 24 to 64 per SM 2 to 8 % slower, one exactly resident wave 10 % slower)
-    int64_t groups = ((int64_t)16 * n_sm + (int64_t)gx * n_streams - 1) / ((int64_t)gx * n_streams);
+    // blocks the device keeps resident at once, asked once per device and kernel variant
+    static std::atomic<int> occ_cache[2][kMaxDevices];
+    const bool slot = dp.device >= 0 && dp.device < kMaxDevices;
+    int per_sm = slot ? occ_cache[bf16 ? 1 : 0][dp.device].load(std::memory_order_acquire) : 0;
+    if (per_sm == 0) {
+        e = bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rerotate_kernel<true>, kRopeThreads, 0)
+                 : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rerotate_kernel<false>, kRopeThreads, 0);
+        if (e != cudaSuccess) return e;
+        if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+        if (slot) occ_cache[bf16 ? 1 : 0][dp.device].store(per_sm, std::memory_order_release);
+    }
+    // As many blocks as fit in kRopeWaves resident waves, not more: each block reuses its angles
+    // over a group of planes, later waves even out SMs of different speed, and a grid that ends
+    // just under a whole number of waves leaves no thin last wave (measured: grids of 2.0x and
+    // 3.5x the resident blocks are 4-8 % slower than 2.7-2.9x; one exactly resident wave with
+    // equal static shares 10 % slower).
+    const int64_t resident = (int64_t)dp.n_sm * per_sm;
+    int64_t groups = kRopeWaves * resident / ((int64_t)gx * n_streams);
     if (groups < 1) groups = 1;
     if (groups > p.planes_per_stream) groups = p.planes_per_stream;
     RopeParams q = p;

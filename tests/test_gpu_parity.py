@@ -841,7 +841,7 @@ def _ordered16(t):
 @pytest.mark.parametrize("layout", [B.ROPE_HALF, B.ROPE_INTERLEAVED])
 def test_rerotate_keys_matches_oracle(dtype, layout):
     # both sides rotate in fp64 and round once, from fp64, to the 16-bit type: results agree bit
-    # for bit except where the angle's last bits (exp2 on the device, pow in the oracle) put a
+    # for bit except where the last bits of the fp64 value (the device's sincos and fused product) put a
     # value on the other side of a rounding boundary - one unit in the last place, rarely
     S, P, cap, D, thr = 2, 3, 700, 128, 400
     cfg = B.make_config(S, P, 1, D, cap, thr, 0, 0, 0, 16, torch.float32, dtype)
