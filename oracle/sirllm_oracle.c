@@ -16,8 +16,9 @@
  * Every function is pinned by tests/test_oracle_*.py against closed forms, the
  * paper's printed cache example, brute force on tiny caches, a long-double
  * recomputation and invariants.  The end-to-end composition (oracle_step) has no
- * number in the paper to be pinned to beyond those per-part pins: parity unpinned
- * at the level of whole multi-round streams.
+ * number in the paper to be pinned to; it is pinned by seven rounds of Algorithm 1
+ * worked by hand on a four-token cache (tests/golden/algorithm1_hand_trace.txt) and
+ * by the invariants of the multi-round tests.
  */
 #include <math.h>
 #include <stdint.h>

@@ -64,6 +64,14 @@ MUTANTS = {
          "(const char *)src + (size_t)j * (size_t)row_bytes, (size_t)row_bytes);"),
     "round: scores not compacted with the cache":
         ("    memcpy(E, E2, sizeof(float) * (size_t)n_keep);", "    (void)E2;"),
+    "round: tags not compacted with the cache":
+        ("        memcpy(serial, s2, sizeof(int64_t) * (size_t)n_keep);", "        (void)s2;"),
+    "round: only the first plane of a cache is compacted":
+        ("        for (int64_t p = 0; p < n_planes; ++p) {\n            char *plane", "        for (int64_t p = 0; p < 1; ++p) {\n            char *plane"),
+    "round: the V cache is left as it was":
+        ("    for (int c = 0; c < 2; ++c) {\n        if (!caches[c])", "    for (int c = 0; c < 1; ++c) {\n        if (!caches[c])"),
+    "round: new scores appended after the decay":
+        ("    l += T;\n    oracle_decay(E, l, eta);", "    oracle_decay(E, l + T, eta);\n    for (int32_t t = 0; t < T; ++t)\n        E[l + t] = new_e[t];\n    l += T;"),
     "interval policy: interval from the retained size":
         ("    int32_t interval = l / budget;", "    int32_t interval = budget / (l - budget + 1) + 1;"),
     "random policy: round not part of the counter":

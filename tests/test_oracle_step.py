@@ -122,3 +122,45 @@ def test_more_new_tokens_than_budget_evicts_inside_the_round():
     dec = (e.numpy() * np.float32(w.decay)).astype(np.float32)
     cut = np.sort(dec[4:448])[::-1][w.budget - 68 - 1]
     assert (dec[mid.numpy()] >= cut).all()
+
+
+def _read_trace(path):
+    head, rounds = {}, []
+    for line in open(path):
+        f = line.split()
+        if not f or f[0].startswith("#"):
+            continue
+        if f[0] == "round":
+            rounds.append({"new": [float(x) for x in f[1:]]})
+        elif f[0] in ("kept", "tokens"):
+            rounds[-1][f[0]] = [int(x) for x in f[1:]]
+        elif f[0] == "scores":
+            rounds[-1]["scores"] = [float(x) for x in f[1:]]
+        else:
+            head[f[0]] = float(f[1])
+    return head, rounds
+
+
+def test_rounds_worked_by_hand_from_algorithm_1(golden_dir):
+    # seven rounds of Algorithm 1 followed on paper (exact binary scores, decay 0.5): pins the
+    # order append -> decay -> evict, the three index sets, the tie rule, the compaction of
+    # scores, tags and rows, and a round without new tokens
+    head, rounds = _read_trace(f"{golden_dir}/algorithm1_hand_trace.txt")
+    cap, dim = 8, 4
+    s = oracle.Stream(cap, int(head["n_sink"]), int(head["n_recent"]), int(head["budget"]),
+                      int(head["threshold"]), head["decay"],
+                      torch.zeros(2, cap, dim, dtype=torch.float16), torch.zeros(2, cap, dim, dtype=torch.float16))
+    assert len(rounds) == 7
+    for r in rounds:
+        T, l, first = len(r["new"]), s.live_len, int(s.next_serial.value)
+        for t in range(T):                       # the round's rows carry the token's number
+            s.k[:, l + t] = first + t
+            s.v[:, l + t] = -(first + t)
+        keep = s.step(torch.tensor(r["new"], dtype=torch.float32))
+        n = s.live_len
+        assert keep.tolist() == r["kept"]
+        assert s.serial[:n].tolist() == r["tokens"]
+        assert s.E[:n].tolist() == r["scores"]
+        for p in range(2):
+            assert s.k[p, :n, 0].tolist() == [float(x) for x in r["tokens"]]
+            assert s.v[p, :n, dim - 1].tolist() == [-float(x) for x in r["tokens"]]
