@@ -451,6 +451,46 @@ def test_step_host_refused_call_leaves_the_device_untouched():
     assert B.sirllm_status(st.ws) == 0
 
 
+def test_rounds_worked_by_hand_from_algorithm_1_on_the_device(golden_dir):
+    # the seven hand-worked rounds of tests/golden/algorithm1_hand_trace.txt through
+    # sirllm_decay_select + sirllm_compact_kv: expected values come from the file, not from the oracle
+    from test_oracle_step import _read_trace
+    head, rounds = _read_trace(f"{golden_dir}/algorithm1_hand_trace.txt")
+    cap, D, P = 8, 8, 3
+    cfg = B.make_config(1, P, 1, D, cap, int(head["budget"]), int(head["n_sink"]), int(head["n_recent"]),
+                        4, 16, torch.float32, torch.float16, threshold=int(head["threshold"]))
+    ws = B.new_workspace(cfg)
+    scores = torch.zeros(1, cap, device=DEV)
+    serial = torch.full((1, cap), -1, dtype=torch.int64, device=DEV)
+    live = torch.zeros(1, dtype=torch.int32, device=DEV)
+    decay = torch.tensor([head["decay"]], device=DEV)
+    keep = torch.zeros(1, cfg.threshold, dtype=torch.int32, device=DEV)
+    n_keep = torch.zeros(1, dtype=torch.int32, device=DEV)
+    k = torch.zeros(1, P, cap, D, dtype=torch.float16, device=DEV)
+    v = torch.zeros_like(k)
+    nxt = 0
+    for r in rounds:
+        T, l = len(r["new"]), int(live[0])
+        for t in range(T):
+            scores[0, l + t] = r["new"][t]
+            serial[0, l + t] = nxt
+            k[0, :, l + t] = nxt
+            v[0, :, l + t] = -nxt
+            nxt += 1
+        live[0] = l + T
+        B.sirllm_decay_select(cfg, scores, serial, live, decay, keep, n_keep, True, ws)
+        B.sirllm_compact_kv(cfg, k, v, k, v, keep, n_keep, ws)
+        n = int(n_keep[0])
+        assert int(live[0]) == n == len(r["kept"])
+        assert keep[0, :n].tolist() == r["kept"]
+        assert serial[0, :n].tolist() == r["tokens"]
+        assert scores[0, :n].tolist() == r["scores"]
+        for p in range(P):
+            assert k[0, p, :n, 0].tolist() == [float(x) for x in r["tokens"]]
+            assert v[0, p, :n, D - 1].tolist() == [-float(x) for x in r["tokens"]]
+    assert B.sirllm_status(ws) == 0
+
+
 def test_step_overflowing_round_is_skipped_and_flagged():
     w = wl.WORKLOADS["tiny"].scaled(n_streams=2, n_layers=1, n_kv_heads=1, capacity=300, budget=256,
                                     new_tokens=200, vocab=1000)
