@@ -53,6 +53,23 @@ def test_score_ragged_vocabularies_and_strides(dtype, V, stride):
     assert_entropy_close(out, oracle.score(buf[:, :V], ids))
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_score_rows_of_a_million_logits(dtype):
+    # a row far wider than any model's vocabulary: dozens of CTAs reduce one row and the last one
+    # to arrive combines their pairs; odd width, odd stride, targets in the first, a middle and
+    # the last column, and one id that has no prediction
+    T, V, stride = 5, 1_000_003, 1_000_011
+    g = torch.Generator().manual_seed(5)
+    buf = (torch.randn(T, stride, generator=g) * 2.5).to(dtype)
+    ids = torch.tensor([0, V // 2, V - 1, -1, 12345], dtype=torch.int32)
+    cfg = _score_cfg(T, V, dtype, stride)
+    ws = B.new_workspace(cfg)
+    out = torch.full((T,), -1.0, device=DEV)
+    B.sirllm_score(cfg, buf.to(DEV)[:, :V], ids.to(DEV), None, out, ws)
+    assert_entropy_close(out, oracle.score(buf[:, :V], ids))
+    assert float(out[3]) == 0.0 and B.sirllm_status(ws) == 0
+
+
 def test_score_closed_forms_on_device():
     import math
     V = 32000
