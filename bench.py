@@ -14,7 +14,8 @@ it starts itself, one per GPU.
 Timing: CUDA events on the launching stream, barrier + synchronize on both sides, max over
 ranks.  The K timed rounds run back to back; every round reads a logits tensor (>= 1 GB on
 the default workload) and a K/V cache (>= 2 GB) far larger than the 126 MB L2, and
-alternates between two logits tensors, so nothing it needs is cache resident.
+rotates through as many logits tensors as it takes to hold twice the L2 (two on the default
+workload, dozens on the workloads with short rounds), so nothing it needs is cache resident.
 """
 from __future__ import annotations
 
@@ -149,8 +150,8 @@ class Pass:
         self.v = torch.zeros(S, P, C, D, dtype=w.torch_kv_dtype, device=dev)
         self.n_new = torch.full((S,), M, dtype=torch.int32, device=dev)
         bias = wl.zipf_bias_table(w.vocab, w.zipf_bias, dev) if w.zipf_bias else None
-        self.pool = []                    # two rounds of logits / ids to alternate between
-        for r in range(2):
+        self.pool = []                    # rounds of logits / ids to rotate through
+        for r in range(logits_pool_size(w)):
             lg = torch.empty(S * M, w.vocab, dtype=w.torch_logits_dtype, device=dev)
             ids = torch.empty(S * M, dtype=torch.int32, device=dev)
             for s in range(S):
@@ -178,7 +179,7 @@ class Pass:
         self.next_serial += T
 
     def step(self, events=None):
-        which = self.round & 1
+        which = self.round % len(self.pool)
         self.round += 1
         if events is None:
             self.fused[which]()
@@ -217,6 +218,17 @@ def step_bytes(w: wl.Workload, moved_rows: int) -> dict:
     return {"score": score, "select": select, "compact": compact, "step": score + select + compact}
 
 
+L2_BYTES = 126 << 20
+
+
+def logits_pool_size(w: wl.Workload) -> int:
+    """Logits tensors the timed rounds rotate through: at least two, and as many as it takes
+    for the pool to hold twice the L2, so that no round finds its logits cache resident."""
+    es = 4 if w.logits_dtype == "f32" else 2
+    per_round = w.n_streams * w.new_tokens * w.vocab * es
+    return max(2, min(96, -(-2 * L2_BYTES // per_round)))
+
+
 def config_dict(w: wl.Workload, world: int, graph: bool = False) -> dict:
     return {"workload": w.name, "streams_per_gpu": w.n_streams,
             "new_tokens_per_round": w.new_tokens, "vocab": w.vocab,
@@ -224,7 +236,8 @@ def config_dict(w: wl.Workload, world: int, graph: bool = False) -> dict:
             "planes": 2 * w.planes_per_stream, "head_dim": w.head_dim,
             "capacity": w.capacity, "budget": w.budget, "n_sink": w.n_sink,
             "n_recent": w.n_recent, "decay": w.decay, "parallelism": f"streams x{world}",
-            "l2": "inputs larger than L2 (logits alternate between two tensors)",
+            "l2": f"inputs larger than L2 (logits rotate through {logits_pool_size(w)} tensors, "
+                  f"K/V cache of {2 * w.n_streams * w.planes_per_stream * w.capacity * w.head_dim * 2 >> 20} MiB)",
             "cuda_graph": graph}
 
 
@@ -256,7 +269,7 @@ def run_ours(args, rank, world, local_rank):
     sync()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     graph = None
-    if args.graph:       # two rounds (one per logits tensor) captured once, replayed K/2 times
+    if args.graph:       # two rounds (two of the logits tensors) captured once, replayed K/2 times
         assert args.steps % 2 == 0, "--graph needs an even --steps"
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
@@ -360,7 +373,7 @@ def run_extras(p: Pass, args):
     tile = 128
     n_tiles = (w.vocab + tile - 1) // tile
     pools = []
-    for lg, ids in p.pool:                       # what an LM-head epilogue would hand over
+    for lg, ids in p.pool[:2]:                   # what an LM-head epilogue would hand over
         rows = lg.shape[0]
         pairs = torch.empty(rows, n_tiles, 2, dtype=torch.float32, device=p.dev)
         for r0 in range(0, rows, 512):
@@ -408,7 +421,7 @@ def run_e2e(p: Pass, args, dist, world):
     w, B, cfg = p.w, p.B, p.cfg
     S, P, M, D = w.n_streams, w.planes_per_stream, w.new_tokens, w.head_dim
     pin = lambda t: t.cpu().pin_memory()
-    h_pool = [(pin(lg), pin(ids)) for lg, ids in p.pool]
+    h_pool = [(pin(lg), pin(ids)) for lg, ids in p.pool[:2]]
     serials = torch.arange(M, device=p.dev)
     h_k = torch.empty(S, P, M, D, dtype=w.torch_kv_dtype).pin_memory()
     h_v = torch.empty(S, P, M, D, dtype=w.torch_kv_dtype).pin_memory()
